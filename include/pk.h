@@ -1,0 +1,167 @@
+/*
+ * pk.h -- C ABI of the packed-attention library for NVIDIA B200 (sm_100a).
+ *
+ * The library evaluates causal self-attention over a PACKED token stream: several
+ * examples are concatenated into one sequence of T tokens, `position_ids` restart at
+ * every example (Sec. 3 "Packing with Position IDs", Sec. 3.1), and every token
+ * attends only to earlier tokens of its own example (Table 1, "Correct
+ * Cross-Attention").  Example boundaries are recovered on the device from the
+ * position ids (paragraph after Table 1: "compute cu_seq_len from position_ids").
+ *
+ * Conventions that hold for every call
+ *   - All data pointers are DEVICE pointers unless the comment says "host".
+ *   - Tensors are contiguous, row-major: q/out/dout/dq are [T, Hq, D]; k/v/dk/dv are
+ *     [T, Hkv, D]; lse is [Hq, T] fp32.  Tensor pointers must be 16-byte aligned.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ *     Everything is enqueued on it; no call synchronises except pk_status_read.
+ *   - The caller owns every buffer.  The library allocates no device memory.
+ *   - Return value: PK_OK or one of the host-detected PK_ERR_* codes.  Problems only
+ *     the device can see (negative position ids, a pipeline wait that ran out) are
+ *     recorded in the workspace's status word; the kernels then stop early and leave
+ *     the outputs untouched.  Read it with pk_status_read.
+ *   - Supported shapes: D in {64, 128}; Hq % Hkv == 0; 0 <= T; T*Hq*D < 2^31.
+ *   - Query head h reads kv head h / (Hq / Hkv).
+ *   - Values of OTHER examples must be finite: a masked probability is exactly 0, but
+ *     0 * Inf is NaN inside a tensor-core contraction.
+ */
+#ifndef PK_H_
+#define PK_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* ---- return / status codes ------------------------------------------------------- */
+#define PK_OK               0
+#define PK_ERR_INVALID_ARG  1   /* null pointer, negative size, misaligned pointer      */
+#define PK_ERR_UNSUPPORTED  2   /* head_dim / head counts / dtype outside the supported set */
+#define PK_ERR_WORKSPACE    3   /* workspace smaller than pk_workspace_bytes            */
+#define PK_ERR_CUDA         4   /* a CUDA runtime/driver call or launch failed          */
+#define PK_ERR_BAD_POSIDS   5   /* device: a position id is negative (detail = index)   */
+#define PK_ERR_TIMEOUT      6   /* device: a bounded pipeline wait ran out (detail = which) */
+#define PK_ERR_NO_PLAN      7   /* device: reuse_plan=1 but the workspace holds no plan for this T */
+
+/* ---- element types of outputs ---------------------------------------------------- */
+#define PK_BF16 0
+#define PK_F32  1
+
+/* ---- workspace sections (pk_workspace_section) ----------------------------------- */
+#define PK_WS_HEADER     0   /* int32[32]: see PK_HDR_* indices                        */
+#define PK_WS_FWD_ITEMS  1   /* int32[T][4]  (q_start, q_len, kv_start, kv_len)        */
+#define PK_WS_BWD_ITEMS  2   /* int32[T][4]  (kv_start, kv_len, q_start, q_len)        */
+#define PK_WS_FWD_ORDER  3   /* int32[T]     item indices, longest work first          */
+#define PK_WS_BWD_ORDER  4   /* int32[T]                                                */
+#define PK_WS_DELTA      5   /* fp32 [Hq][T] row sums of dO*O                           */
+#define PK_WS_DQ_ACC     6   /* fp32 [T+128][Hq][D] accumulator of dQ                   */
+#define PK_WS_ROPE_TABLE 7   /* fp32 [T][D/2][2] (cos, sin) of pos * theta^(-2i/D)      */
+#define PK_WS_NUM_SECTIONS 8
+
+/* indices into the int32 header */
+#define PK_HDR_STATUS      0
+#define PK_HDR_DETAIL      1
+#define PK_HDR_N_EXAMPLES  2
+#define PK_HDR_MAX_SEQLEN  3
+#define PK_HDR_N_ITEMS     4   /* forward and backward lists have the same length      */
+#define PK_HDR_PLAN_T      5   /* T the plan was built for, -1 if none                  */
+
+/*
+ * Tile shape used by the work lists (rows of a query block, rows of a key block).
+ * Not in the paper: the lists are how "tiles outside an example's causal block are
+ * never scheduled" is made checkable.  Host pointers.  Always returns PK_OK.
+ */
+int pk_tile_shape(int32_t* bm, int32_t* bn);
+
+/*
+ * Bytes of workspace the other calls need for a stream of T tokens (upper bound over
+ * every example layout).  Returns 0 for unsupported arguments.
+ */
+size_t pk_workspace_bytes(int32_t T, int32_t Hq, int32_t Hkv, int32_t D);
+
+/*
+ * Byte offset and size of one section of the workspace (PK_WS_*), so that a caller or
+ * a test can look at the plan.  Host pointers.  PK_ERR_INVALID_ARG for a bad section.
+ */
+int pk_workspace_section(int32_t which, int32_t T, int32_t Hq, int32_t Hkv, int32_t D,
+                         size_t* offset, size_t* bytes);
+
+/*
+ * Boundary recovery and planning (paragraph after Table 1; Sec. 3.1 for the form of
+ * the ids).  Token t starts an example iff t == 0 or position_ids[t] <= position_ids[t-1].
+ *   position_ids  int32 [T]
+ *   cu_seqlens    int32 [T+1] out: the E start offsets, then T, then T in every
+ *                 remaining entry
+ *   n_examples    int32 [1] out (device): E
+ *   max_seqlen    int32 [1] out (device): longest example
+ *   workspace     >= pk_workspace_bytes(T, Hq, Hkv, D) bytes, 256-byte aligned.  Receives the
+ *                 plan: forward items (a block of <= bm query rows of one example and
+ *                 the key range [example start, last row] it may see), backward items
+ *                 (a block of <= bn key rows and the query range up to the example end
+ *                 that may see it), both in ascending (example, block) order, plus for
+ *                 each list the stable permutation by descending number of tiles.
+ * T == 0 is valid: cu_seqlens = [0], E = 0.  No host round trip; one kernel launch.
+ */
+int pk_seqlens_from_posids(const int32_t* position_ids, int32_t T,
+                           int32_t* cu_seqlens, int32_t* n_examples, int32_t* max_seqlen,
+                           void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Rotary embedding indexed by position_ids, in place (unfused form of what the
+ * attention calls do while loading Q/K tiles).  The paper only requires that models
+ * "expose position IDs" (end of Sec. 3.5); the rotation is the usual one:
+ * pairs (i, i + D/2), angle position_ids[t] * theta^(-2i/D); inverse != 0 rotates by
+ * the negative angle.   x: bf16 [T, H, D].  D even, <= 256.
+ */
+int pk_rope_apply(void* x, const int32_t* position_ids, int32_t T, int32_t H, int32_t D,
+                  float theta, int32_t inverse, void* stream);
+
+/*
+ * Forward (Sec. 3, Table 1 "Correct Cross-Attention"): for every query head h and
+ * token i of example e,  S_ij = softmax_scale * <q'_i, k'_j> for s_e <= j <= i,
+ * lse[h][i] = log sum_j exp S_ij (natural log),  out[i][h] = sum_j exp(S_ij - lse) v_j.
+ *   q, k, v       bf16
+ *   rope_theta    > 0: q and k are rotated by position_ids while their tiles are loaded
+ *                 (q', k'); <= 0: q and k are used as given
+ *   out           [T, Hq, D], element type out_dtype (PK_BF16 or PK_F32)
+ *   lse           fp32 [Hq, T]
+ *   reuse_plan    0: run the planning step of pk_seqlens_from_posids first (same stream);
+ *                 1: use the plan already in `workspace` (must be for these position_ids)
+ */
+int pk_attn_fwd(const void* q, const void* k, const void* v, const int32_t* position_ids,
+                int32_t T, int32_t Hq, int32_t Hkv, int32_t D,
+                float softmax_scale, float rope_theta,
+                void* out, int32_t out_dtype, float* lse,
+                int32_t reuse_plan, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Backward of pk_attn_fwd: given dout = dL/dout, computes dq, dk, dv.  A row-sum
+ * pre-pass forms delta = sum_d dout*out; the main kernel recomputes the probabilities
+ * from lse, dV = P^T dO, dP = dO V^T, dS = P o (dP - delta), dQ = scale dS K',
+ * dK = scale dS^T Q'; dK and dV are summed over the Hq/Hkv query heads of a kv head.
+ * With rope_theta > 0 the gradients are with respect to the un-rotated q and k.
+ *   out, out_dtype   the forward's output as it was written
+ *   dq [T,Hq,D], dk, dv [T,Hkv,D]   element type grad_dtype (PK_BF16 or PK_F32)
+ * dV and dK rows are accumulated in a fixed order (bitwise reproducible); dQ is
+ * accumulated with floating-point atomics (order not fixed).
+ */
+int pk_attn_bwd(const void* dout, const void* q, const void* k, const void* v,
+                const void* out, int32_t out_dtype, const float* lse,
+                const int32_t* position_ids,
+                int32_t T, int32_t Hq, int32_t Hkv, int32_t D,
+                float softmax_scale, float rope_theta,
+                void* dq, void* dk, void* dv, int32_t grad_dtype,
+                int32_t reuse_plan, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Copies the workspace's status word to the host and waits for `stream` (the only call
+ * that synchronises).  code/detail are host pointers: PK_OK, or the first device-side
+ * error recorded since the last planning step.
+ */
+int pk_status_read(const void* workspace, void* stream, int32_t* code, int32_t* detail);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PK_H_ */

@@ -1,0 +1,37 @@
+// Small host-only entry points of the C ABI: tile shape, workspace sizing and layout,
+// status read-back.
+#include "pk_common.cuh"
+
+extern "C" int pk_tile_shape(int32_t* bm, int32_t* bn) {
+  if (bm) *bm = pk::kBM;
+  if (bn) *bn = pk::kBN;
+  return PK_OK;
+}
+
+extern "C" size_t pk_workspace_bytes(int32_t T, int32_t Hq, int32_t Hkv, int32_t D) {
+  if (!pk::shape_supported(T, Hq, Hkv, D)) return 0;
+  return pk::workspace_layout(T, Hq, Hkv, D).total;
+}
+
+extern "C" int pk_workspace_section(int32_t which, int32_t T, int32_t Hq, int32_t Hkv, int32_t D,
+                                    size_t* offset, size_t* bytes) {
+  if (which < 0 || which >= PK_WS_NUM_SECTIONS || offset == nullptr || bytes == nullptr)
+    return PK_ERR_INVALID_ARG;
+  if (!pk::shape_supported(T, Hq, Hkv, D)) return PK_ERR_UNSUPPORTED;
+  const pk::WorkspaceLayout lay = pk::workspace_layout(T, Hq, Hkv, D);
+  *offset = lay.off[which];
+  *bytes = lay.bytes[which];
+  return PK_OK;
+}
+
+extern "C" int pk_status_read(const void* workspace, void* stream, int32_t* code, int32_t* detail) {
+  if (workspace == nullptr || code == nullptr || detail == nullptr) return PK_ERR_INVALID_ARG;
+  int32_t host[2] = {0, 0};
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (cudaMemcpyAsync(host, workspace, sizeof(host), cudaMemcpyDeviceToHost, s) != cudaSuccess)
+    return PK_ERR_CUDA;
+  if (cudaStreamSynchronize(s) != cudaSuccess) return PK_ERR_CUDA;
+  *code = host[PK_HDR_STATUS];
+  *detail = host[PK_HDR_DETAIL];
+  return PK_OK;
+}

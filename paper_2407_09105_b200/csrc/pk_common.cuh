@@ -1,0 +1,90 @@
+// Shared host/device definitions of the packed-attention library: workspace layout,
+// status word, launch-error helper.  No attention arithmetic lives here.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "pk.h"
+
+namespace pk {
+
+constexpr int kBM = 128;   // query rows per tile
+constexpr int kBN = 128;   // key rows per tile
+constexpr int kHeaderInts = 32;
+
+// header slots beyond the public PK_HDR_* ones
+constexpr int kHdrFwdTicket = 8;
+constexpr int kHdrBwdTicket = 9;
+
+struct WorkspaceLayout {
+  size_t off[PK_WS_NUM_SECTIONS];
+  size_t bytes[PK_WS_NUM_SECTIONS];
+  size_t off_cu;         // int32 [T+1]   the plan's own copy of cu_seqlens
+  size_t off_ex_base;    // int32 [T+2]   first item index of every example
+  size_t off_hist;       // int32 [2][T/128 + 4] counting-sort cursors (fwd, bwd)
+  size_t hist_stride;    // ints per histogram
+  size_t plan_total;     // bytes of the part that depends on T only
+  size_t total;
+};
+
+__host__ __device__ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+__host__ inline WorkspaceLayout workspace_layout(int64_t T, int64_t Hq, int64_t Hkv, int64_t D) {
+  WorkspaceLayout w;
+  size_t cur = 0;
+  auto put = [&](int which, size_t bytes) {
+    w.off[which] = cur;
+    w.bytes[which] = bytes;
+    cur = align_up(cur + bytes, 256);
+  };
+  const size_t Tn = (size_t)(T > 0 ? T : 1);
+  // plan part: depends on T only
+  put(PK_WS_HEADER, sizeof(int32_t) * kHeaderInts);
+  put(PK_WS_FWD_ITEMS, sizeof(int32_t) * 4 * Tn);
+  put(PK_WS_BWD_ITEMS, sizeof(int32_t) * 4 * Tn);
+  put(PK_WS_FWD_ORDER, sizeof(int32_t) * Tn);
+  put(PK_WS_BWD_ORDER, sizeof(int32_t) * Tn);
+  w.off_cu = cur;
+  cur = align_up(cur + sizeof(int32_t) * (Tn + 1), 256);
+  w.off_ex_base = cur;
+  cur = align_up(cur + sizeof(int32_t) * (Tn + 2), 256);
+  w.hist_stride = Tn / 128 + 4;
+  w.off_hist = cur;
+  cur = align_up(cur + sizeof(int32_t) * 2 * w.hist_stride, 256);
+  w.plan_total = cur;
+  // attention part: depends on the head shape
+  put(PK_WS_DELTA, sizeof(float) * (size_t)Hq * Tn);
+  put(PK_WS_DQ_ACC, sizeof(float) * (size_t)(T + 128) * (size_t)Hq * (size_t)D);
+  put(PK_WS_ROPE_TABLE, sizeof(float) * 2 * Tn * (size_t)(D / 2));
+  w.total = cur;
+  (void)Hkv;
+  return w;
+}
+
+inline bool shape_supported(int32_t T, int32_t Hq, int32_t Hkv, int32_t D) {
+  if (T < 0 || Hq <= 0 || Hkv <= 0) return false;
+  if (D != 64 && D != 128) return false;
+  if (Hq % Hkv != 0) return false;
+  if ((int64_t)T * Hq * D >= ((int64_t)1 << 31)) return false;
+  return true;
+}
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Records the first device-side error; later ones are dropped.
+__device__ inline void set_status(int32_t* header, int32_t code, int32_t detail) {
+  if (atomicCAS(&header[PK_HDR_STATUS], PK_OK, code) == PK_OK) header[PK_HDR_DETAIL] = detail;
+}
+
+inline int launch_status() { return cudaGetLastError() == cudaSuccess ? PK_OK : PK_ERR_CUDA; }
+
+// internal entry points shared between translation units
+int plan_launch(const int32_t* position_ids, int32_t T, int32_t* cu_seqlens, int32_t* n_examples,
+                int32_t* max_seqlen, void* workspace, const WorkspaceLayout& lay,
+                cudaStream_t stream);
+int rope_table_launch(const int32_t* position_ids, int32_t T, int32_t D, float theta,
+                      float* table, cudaStream_t stream);
+
+}  // namespace pk

@@ -1,0 +1,81 @@
+// Rotary embedding indexed by position_ids: the standalone in-place kernel and the
+// (cos, sin) table the attention kernels read while they rotate Q/K tiles in shared
+// memory.  The paper requires only that position ids reach the attention (end of
+// Sec. 3.5); the rotation is the usual half-split one.  Angles are formed in fp64 so
+// that ids up to 2^17 lose nothing before the fp32 cos/sin are taken.
+#include <cuda_bf16.h>
+
+#include "pk_common.cuh"
+
+namespace pk {
+namespace {
+
+__device__ __forceinline__ void angle_cos_sin(int pos, int i, int D, double log2_theta,
+                                              float* c, float* s) {
+  const double inv_freq = exp2(-2.0 * (double)i / (double)D * log2_theta);
+  double sd, cd;
+  sincos((double)pos * inv_freq, &sd, &cd);
+  *c = (float)cd;
+  *s = (float)sd;
+}
+
+// table[t][i] = (cos, sin)(pos[t] * theta^(-2i/D))
+__global__ void rope_table_kernel(const int32_t* __restrict__ pos, int T, int D, double log2_theta,
+                                  float2* __restrict__ table) {
+  const int half = D / 2;
+  const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= (int64_t)T * half) return;
+  const int t = (int)(idx / half), i = (int)(idx % half);
+  float c, s;
+  angle_cos_sin(pos[t], i, D, log2_theta, &c, &s);
+  table[idx] = make_float2(c, s);
+}
+
+// One thread per (token, pair index); loops over heads so cos/sin are formed once.
+__global__ void rope_apply_kernel(__nv_bfloat16* __restrict__ x, const int32_t* __restrict__ pos,
+                                  int T, int H, int D, double log2_theta, int inverse) {
+  const int half = D / 2;
+  const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= (int64_t)T * half) return;
+  const int t = (int)(idx / half), i = (int)(idx % half);
+  float c, s;
+  angle_cos_sin(pos[t], i, D, log2_theta, &c, &s);
+  if (inverse) s = -s;
+  __nv_bfloat16* row = x + (int64_t)t * H * D;
+  for (int h = 0; h < H; ++h) {
+    const float a = __bfloat162float(row[h * D + i]);
+    const float b = __bfloat162float(row[h * D + i + half]);
+    row[h * D + i] = __float2bfloat16_rn(a * c - b * s);
+    row[h * D + i + half] = __float2bfloat16_rn(b * c + a * s);
+  }
+}
+
+}  // namespace
+
+int rope_table_launch(const int32_t* position_ids, int32_t T, int32_t D, float theta,
+                      float* table, cudaStream_t stream) {
+  if (T == 0) return PK_OK;
+  const int64_t n = (int64_t)T * (D / 2);
+  const int threads = 256;
+  const unsigned blocks = (unsigned)((n + threads - 1) / threads);
+  rope_table_kernel<<<blocks, threads, 0, stream>>>(position_ids, T, D, log2((double)theta),
+                                                    reinterpret_cast<float2*>(table));
+  return launch_status();
+}
+
+}  // namespace pk
+
+extern "C" int pk_rope_apply(void* x, const int32_t* position_ids, int32_t T, int32_t H,
+                             int32_t D, float theta, int32_t inverse, void* stream) {
+  if (T < 0 || H <= 0) return PK_ERR_INVALID_ARG;
+  if (D <= 0 || D > 256 || (D & 1)) return PK_ERR_UNSUPPORTED;
+  if (!(theta > 0.0f)) return PK_ERR_INVALID_ARG;
+  if (T == 0) return PK_OK;
+  if (x == nullptr || position_ids == nullptr) return PK_ERR_INVALID_ARG;
+  const int64_t n = (int64_t)T * (D / 2);
+  const int threads = 256;
+  const unsigned blocks = (unsigned)((n + threads - 1) / threads);
+  pk::rope_apply_kernel<<<blocks, threads, 0, static_cast<cudaStream_t>(stream)>>>(
+      static_cast<__nv_bfloat16*>(x), position_ids, T, H, D, log2((double)theta), inverse);
+  return pk::launch_status();
+}
