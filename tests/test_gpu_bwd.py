@@ -1,0 +1,94 @@
+"""GPU parity of the backward against the fp64 oracle (same seeded bf16 inputs).
+
+Tolerance: max-abs 2e-2 on fp32 gradients; bf16 gradients get half a bf16 ulp of the
+exact value on top (2e-2 + 2^-8 |ref|).  The forward output handed to the backward is
+the GPU's own (fp32), as in training."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import packed_attention as orc
+from paper_2407_09105_b200 import api, workloads as wl
+from helpers import f64, max_abs, run_bwd, run_fwd, to_cuda
+
+pytestmark = pytest.mark.gpu
+
+TOL_G = 2e-2
+
+
+def _case(lens, Hq, Hkv, D, theta, seed=0, grad_dtype=torch.float32, out_dtype=torch.float32,
+          offsets=None):
+    w = wl.Workload("t", seed, Hq, Hkv, D, theta, [list(lens)], "test")
+    st = to_cuda(wl.stream_tensors(w, list(lens), 0, "cpu", offsets))
+    out, lse, ws = run_fwd(st, w, out_dtype)
+    dq, dk, dv = run_bwd(st, w, out, lse, ws, grad_dtype)
+    edq, edk, edv = orc.attn_bwd(f64(st.dout), f64(st.q), f64(st.k), f64(st.v),
+                                 st.position_ids.cpu().numpy(), w.softmax_scale, theta)
+    errs = {}
+    for name, g, e in (("dq", dq, edq), ("dk", dk, edk), ("dv", dv, edv)):
+        g = f64(g)
+        assert not np.isnan(g).any(), name
+        if grad_dtype == torch.float32:
+            assert max_abs(g, e) <= TOL_G, (name, max_abs(g, e))
+        else:
+            assert (np.abs(g - e) <= TOL_G + 2.0 ** -8 * np.abs(e)).all(), (name, max_abs(g, e))
+        errs[name] = max_abs(g, e)
+    return errs
+
+
+def test_c1_tiny_pack():
+    w = wl.workload("c1")
+    _case(w.streams[0], w.num_q_heads, w.num_kv_heads, w.head_dim, w.rope_theta)
+
+
+@pytest.mark.parametrize("D", [64, 128])
+@pytest.mark.parametrize("lens", [[1], [128], [129], [127, 1, 130], [300, 5, 5, 700, 1]])
+def test_tile_edges(D, lens):
+    _case(lens, 2, 2, D, 0.0, seed=3)
+
+
+@pytest.mark.parametrize("D", [64, 128])
+def test_gqa(D):
+    _case([200, 77, 400], 8, 2, D, 0.0, seed=4)
+
+
+@pytest.mark.parametrize("D,theta", [(64, 1e4), (128, 1e4), (128, 5e5)])
+def test_fused_rope(D, theta):
+    _case([150, 260, 3, 129], 4, 2, D, theta, seed=5)
+
+
+def test_rope_fragment_ids():
+    _case([100, 50], 2, 2, 128, 1e4, seed=6, offsets=[1000, 0])
+
+
+def test_bf16_grads_and_bf16_forward_output():
+    _case([300, 5, 200], 4, 2, 128, 0.0, seed=7, grad_dtype=torch.bfloat16,
+          out_dtype=torch.bfloat16)
+    _case([300, 5, 200], 4, 4, 64, 1e4, seed=7, grad_dtype=torch.bfloat16,
+          out_dtype=torch.bfloat16)
+
+
+def test_long_example_many_tiles():
+    _case([2100, 37], 2, 1, 128, 0.0, seed=8)
+
+
+def test_fused_rope_equals_unfused_composition():
+    """Gradients with fused RoPE are with respect to the un-rotated q and k: they equal
+    rotate -> attention without RoPE -> rotate the gradients back."""
+    lens, Hq, Hkv, D, theta = [140, 90], 4, 2, 128, 1e4
+    w = wl.Workload("t", 9, Hq, Hkv, D, theta, [lens], "test")
+    st = to_cuda(wl.stream_tensors(w, lens, 0, "cpu"))
+    out, lse, ws = run_fwd(st, w)
+    dq, dk, dv = run_bwd(st, w, out, lse, ws)
+    qr, kr = st.q.clone(), st.k.clone()
+    api.pk_rope_apply(qr, st.position_ids, theta)
+    api.pk_rope_apply(kr, st.position_ids, theta)
+    st2 = wl.StreamTensors(st.position_ids, qr, kr, st.v, st.dout, lens)
+    out2, lse2, ws2 = run_fwd(st2, w, theta=0.0)
+    assert torch.equal(out, out2) and torch.equal(lse, lse2)
+    dq2, dk2, dv2 = run_bwd(st2, w, out2, lse2, ws2, theta=0.0)
+    assert torch.equal(dv, dv2)
+    # rotate the unfused gradients back in fp64 on the host (the kernel does it in fp32)
+    pos = st.position_ids.cpu().numpy()
+    assert max_abs(f64(dq), orc.rope(f64(dq2), pos, theta, inverse=True)) < 1e-3
+    assert max_abs(f64(dk), orc.rope(f64(dk2), pos, theta, inverse=True)) < 1e-3
