@@ -1,0 +1,347 @@
+#!/usr/bin/env python
+"""Benchmark of the packed-attention hot path on B200.
+
+One step = one pass of the whole path over one packed stream: plan (position_ids ->
+cu_seqlens + work lists), forward, delta pre-pass, backward, dQ finishing pass.
+Default workload: c4, the Mistral-7B-shaped GQA layer (32 q / 8 kv heads, head_dim 128)
+over 16 first-fit-decreasing bins of 8192 tokens, run as one flat stream (bin edges are
+example edges, so the result is identical to 16 separate calls).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c4] [--impl reference]
+
+Prints ONE JSON line.  `value` is useful TFLOP/s: 14 * D * Hq * sum_e L_e (L_e + 1) / 2
+floating-point operations per step (forward 4, backward 10 per causal pair and head
+dimension) divided by the device time of the step.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2407_09105_b200 import workloads as wl  # noqa: E402
+
+METRIC = "packed_attn_fwd_bwd_useful_tflops"
+UNIT = "TFLOP/s"
+
+# DRAM bytes per causal (query, key, q-head) pair of the backward main kernel, from the ncu
+# capture summarised in profiles/ (scaled to a launch by the number of pairs); None = not captured.
+NCU_BWD_DRAM_BYTES_PER_PAIR = None
+
+
+def _peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"burst": float(p["bf16_tflops"]), "sustained": float(p["bf16_tflops_sustained"]),
+                "hbm_gbs": float(p["hbm_gbs"]), "source": "measured"}
+    return {"burst": 1590.0, "sustained": 1400.0, "hbm_gbs": 6650.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.samples = []
+        self.proc = None
+        self.thread = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread.start()
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.samples.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for s in self.samples:
+            parts = [x.strip() for x in s.split(",")]
+            if len(parts) < 6:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, parts[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": float(np.median(sm)) if sm else None,
+                "sm_max_mhz": float(max(mx)) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def _oracle_sample(w: wl.Workload):
+    """A bounded sample of whole examples of the workload for the CPU oracle: the example
+    closest to 2048 tokens plus the eight shortest ones, all heads."""
+    lens = w.flat_lengths()
+    order = sorted(range(len(lens)), key=lambda i: lens[i])
+    mid = min(range(len(lens)), key=lambda i: abs(lens[i] - 2048))
+    pick = sorted(set(order[:8] + [mid]))
+    return [lens[i] for i in pick]
+
+
+def _time_oracle(w: wl.Workload, steps: int = 1):
+    """Runs the fp64 numpy oracle (forward + backward) on the sample; returns
+    (useful TFLOP/s, seconds per pass, threads, description)."""
+    from oracle import packed_attention as orc
+    try:
+        from threadpoolctl import threadpool_info
+        threads = max([p.get("num_threads", 1) for p in threadpool_info()] or [1])
+    except Exception:
+        threads = len(os.sched_getaffinity(0))
+    lens = _oracle_sample(w)
+    sw = wl.Workload(w.name + "_sample", w.seed, w.num_q_heads, w.num_kv_heads, w.head_dim,
+                     w.rope_theta, [lens], w.packing)
+    st = wl.stream_tensors(sw, lens, 0, "cpu")
+    q, k, v, do = (x.to(torch.float64).numpy() for x in (st.q, st.k, st.v, st.dout))
+    pos = st.position_ids.numpy()
+    best = None
+    for _ in range(steps):
+        t0 = time.perf_counter()
+        orc.attn_fwd(q, k, v, pos, sw.softmax_scale, sw.rope_theta)
+        orc.attn_bwd(do, q, k, v, pos, sw.softmax_scale, sw.rope_theta)
+        dt = time.perf_counter() - t0
+        best = dt if best is None else min(best, dt)
+    flops = sw.useful_flops_fwd + sw.useful_flops_bwd
+    desc = (f"{len(lens)} whole examples of {w.name} (lengths {lens}), all {w.num_q_heads} q heads, "
+            f"fwd+bwd in fp64 numpy; {sum(lens)} tokens, {flops / 1e9:.1f} useful GFLOP")
+    return flops / best / 1e12, best, threads, desc, sum(lens)
+
+
+def run_reference(args, w):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    times = []
+    for _ in range(max(1, min(args.warmup, 1))):
+        _time_oracle(w)
+    tf = None
+    for _ in range(max(1, min(args.steps, 3))):
+        tf, dt, threads, desc, toks = _time_oracle(w)
+        times.append(dt)
+    dt = float(np.mean(times))
+    sw_flops = tf * min(times) * 1e12
+    value = sw_flops / dt / 1e12
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": len(times), "warmup": 1, "ms_per_step": dt * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": f"{w.name} ({w.packing}), bounded sample per step", "Hq": w.num_q_heads,
+                   "Hkv": w.num_kv_heads, "head_dim": w.head_dim},
+        "tokens_per_s": toks / dt,
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle",
+                         "sample": desc},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default="c4")
+    ap.add_argument("--impl", default="ours")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl != "reference" else args.warmup
+
+    w = wl.workload(args.workload)
+    if args.impl == "reference":
+        run_reference(args, w)
+        return
+
+    from paper_2407_09105_b200 import api
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist = dist_mod
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    # every rank works on its own replica of the workload (different values, same lengths)
+    lens = w.flat_lengths()
+    st = wl.stream_tensors(w, lens, stream_index=rank, device="cuda")
+    T, Hq, D = st.q.shape
+    Hkv = st.k.shape[1]
+    scale, theta = w.softmax_scale, w.rope_theta
+    ws = api.alloc_workspace(T, Hq, Hkv, D)
+    out = torch.empty_like(st.q)
+    lse = torch.empty((Hq, T), dtype=torch.float32, device="cuda")
+    dq, dk, dv = torch.empty_like(st.q), torch.empty_like(st.k), torch.empty_like(st.v)
+    stream = torch.cuda.current_stream()
+
+    def step():
+        api.pk_attn_fwd(st.q, st.k, st.v, st.position_ids, scale, theta, out, lse, ws,
+                        reuse_plan=False, stream=stream)
+        api.pk_attn_bwd(st.dout, st.q, st.k, st.v, out, lse, st.position_ids, scale, theta,
+                        dq, dk, dv, ws, reuse_plan=True, stream=stream)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        step()
+    code, detail = api.pk_status_read(ws)
+    if code != api.PK_OK:
+        raise SystemExit(f"device status {code} (detail {detail})")
+
+    # per-kernel events: recorded by the library around the two main kernels
+    kev = {k: [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+               for _ in range(args.steps)] for k in (api.PK_KERNEL_FWD, api.PK_KERNEL_BWD)}
+    for pairs in kev.values():
+        for a, b in pairs:
+            a.record(stream)
+            b.record(stream)
+    sampler = ClockSampler(local_rank)
+    barrier()
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for i in range(args.steps):
+        for k, pairs in kev.items():
+            api.pk_set_timing_events(k, pairs[i][0], pairs[i][1])
+        step()
+    e1.record(stream)
+    barrier()
+    clocks = sampler.stop()
+    for k in kev:
+        api.pk_set_timing_events(k, None, None)
+    ms_total = e0.elapsed_time(e1)
+    t_local = torch.tensor([ms_total], dtype=torch.float64, device="cuda")
+    if dist is not None:
+        dist.all_reduce(t_local, op=dist.ReduceOp.MAX)
+    ms_step = float(t_local.item()) / args.steps
+    fwd_ms = float(np.mean([a.elapsed_time(b) for a, b in kev[api.PK_KERNEL_FWD]]))
+    bwd_ms = float(np.mean([a.elapsed_time(b) for a, b in kev[api.PK_KERNEL_BWD]]))
+
+    flops_step = w.useful_flops_fwd + w.useful_flops_bwd
+    value = world * flops_step / (ms_step * 1e-3) / 1e12
+    tokens_per_s = world * T / (ms_step * 1e-3)
+
+    # ---- end to end: host buffers in, host buffers out, through the same calls ------------
+    e2e = None
+    if not args.no_e2e:
+        host_in = [x.cpu().pin_memory() for x in (st.q, st.k, st.v, st.dout, st.position_ids)]
+        dev_in = [st.q, st.k, st.v, st.dout, st.position_ids]
+        dev_out = [out, dq, dk, dv]
+        host_out = [torch.empty(x.shape, dtype=x.dtype, pin_memory=True) for x in dev_out]
+        h2d = sum(x.numel() * x.element_size() for x in host_in)
+        d2h = sum(x.numel() * x.element_size() for x in host_out)
+
+        def e2e_step():
+            for h, d in zip(host_in, dev_in):
+                d.copy_(h, non_blocking=True)
+            step()
+            for d, h in zip(dev_out, host_out):
+                h.copy_(d, non_blocking=True)
+
+        n_e2e = max(3, min(args.steps, 5))
+        e2e_step()
+        barrier()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        for _ in range(n_e2e):
+            e2e_step()
+        b.record(stream)
+        barrier()
+        t = torch.tensor([a.elapsed_time(b)], dtype=torch.float64, device="cuda")
+        if dist is not None:
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_e2e = float(t.item()) / n_e2e
+        e2e = {"value": world * flops_step / (ms_e2e * 1e-3) / 1e12, "unit": UNIT,
+               "ms_per_step": ms_e2e, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    peaks = _peaks()
+    bwd_tflops = w.useful_flops_bwd / (bwd_ms * 1e-3) / 1e12
+    fwd_tflops = w.useful_flops_fwd / (fwd_ms * 1e-3) / 1e12
+    roofline = {
+        "kernel": "attn_bwd_kernel", "bound": "tensor", "achieved": bwd_tflops,
+        "peak": peaks["sustained"], "peak_kind": f"bf16 sustained, {peaks['source']}",
+        "peak_burst": peaks["burst"], "unit": "TFLOP/s", "frac": bwd_tflops / peaks["sustained"],
+        "traffic": (None if NCU_BWD_DRAM_BYTES_PER_PAIR is None
+                    else NCU_BWD_DRAM_BYTES_PER_PAIR * w.causal_pairs * Hq),
+        "ms_per_launch": bwd_ms,
+        "fwd_kernel": {"achieved": fwd_tflops, "frac": fwd_tflops / peaks["sustained"],
+                       "ms_per_launch": fwd_ms},
+    }
+    cpu_baseline = None
+    if not args.no_cpu_baseline:
+        tf, dt, threads, desc, _ = _time_oracle(w)
+        cpu_baseline = {"value": tf, "unit": UNIT, "cores": threads, "kind": "oracle",
+                        "sample": desc, "seconds": dt}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": f"{w.name}: {w.packing}, {len(w.streams)} packs as one flat stream",
+                   "tokens": T, "examples": len(lens), "Hq": Hq, "Hkv": Hkv, "head_dim": D,
+                   "rope_theta": theta, "causal_pairs": w.causal_pairs,
+                   "flop_convention": "14*D*Hq*sum L(L+1)/2", "l2": "inputs_exceed_l2",
+                   "replicas": world},
+        "tokens_per_s": tokens_per_s,
+        "pct_of_bf16_peak": {"sustained": 100 * value / world / peaks["sustained"],
+                             "burst": 100 * value / world / peaks["burst"],
+                             "source": peaks["source"]},
+        "clocks": clocks, "e2e": e2e, "gpu_launches": 5 * args.steps + (2 * args.steps if theta > 0 else 0),
+        "roofline": roofline, "cpu_baseline": cpu_baseline,
+    }
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -161,6 +161,21 @@ int pk_attn_bwd(const void* dout, const void* q, const void* k, const void* v,
  */
 int pk_status_read(const void* workspace, void* stream, int32_t* code, int32_t* detail);
 
+/*
+ * Measurement aid (no counterpart in the paper): asks the library to record the CUDA
+ * events `start` and `stop` (cudaEvent_t passed as void*, owned by the caller) on the
+ * call's stream immediately before and after every later launch of kernel `which`
+ * (PK_KERNEL_*), so that a benchmark can time one kernel inside a multi-kernel call.
+ * Pass NULL for both to stop recording.  Process-wide and not thread-safe.
+ */
+#define PK_KERNEL_PLAN      0
+#define PK_KERNEL_FWD       1
+#define PK_KERNEL_DELTA     2
+#define PK_KERNEL_BWD       3
+#define PK_KERNEL_DQ_FINISH 4
+#define PK_NUM_KERNELS      5
+int pk_set_timing_events(int32_t which, void* start, void* stop);
+
 #ifdef __cplusplus
 }
 #endif

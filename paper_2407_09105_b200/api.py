@@ -45,6 +45,7 @@ _SIGNATURES = {
                                    _i32, _i32, _i32, _i32, _f32, _f32,
                                    _vp, _vp, _vp, _i32, _i32, _vp, _sz, _vp]),
     "pk_status_read": (ctypes.c_int, [_vp, _vp, ctypes.POINTER(_i32), ctypes.POINTER(_i32)]),
+    "pk_set_timing_events": (ctypes.c_int, [_i32, _vp, _vp]),
 }
 
 EXPORTED_SYMBOLS = tuple(_SIGNATURES)
@@ -174,6 +175,18 @@ def pk_status_read(workspace: torch.Tensor, stream=None) -> Tuple[int, int]:
            lib().pk_status_read(_ptr(workspace), _stream(stream), ctypes.byref(code),
                                 ctypes.byref(detail)))
     return code.value, detail.value
+
+
+PK_KERNEL_PLAN, PK_KERNEL_FWD, PK_KERNEL_DELTA, PK_KERNEL_BWD, PK_KERNEL_DQ_FINISH = range(5)
+
+
+def pk_set_timing_events(which: int, start: Optional[torch.cuda.Event],
+                         stop: Optional[torch.cuda.Event]) -> None:
+    """``start``/``stop`` must have been created with ``enable_timing=True`` and recorded
+    once (torch creates the underlying event lazily); ``None`` clears the hook."""
+    s = None if start is None else start.cuda_event
+    e = None if stop is None else stop.cuda_event
+    _check("pk_set_timing_events", lib().pk_set_timing_events(which, s, e))
 
 
 def workspace_view(workspace: torch.Tensor, which: int, T: int, Hq: int, Hkv: int, D: int,

@@ -2,6 +2,17 @@
 // status read-back.
 #include "pk_common.cuh"
 
+namespace pk {
+cudaEvent_t g_timing_events[PK_NUM_KERNELS][2] = {};
+}
+
+extern "C" int pk_set_timing_events(int32_t which, void* start, void* stop) {
+  if (which < 0 || which >= PK_NUM_KERNELS) return PK_ERR_INVALID_ARG;
+  pk::g_timing_events[which][0] = static_cast<cudaEvent_t>(start);
+  pk::g_timing_events[which][1] = static_cast<cudaEvent_t>(stop);
+  return PK_OK;
+}
+
 extern "C" int pk_tile_shape(int32_t* bm, int32_t* bn) {
   if (bm) *bm = pk::kBM;
   if (bn) *bn = pk::kBN;

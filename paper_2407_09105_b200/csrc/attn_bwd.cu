@@ -471,6 +471,7 @@ int launch_bwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& 
   int32_t* hdr = reinterpret_cast<int32_t*>(ws + lay.off[PK_WS_HEADER]);
   if (cudaMemsetAsync(hdr + kHdrBwdTicket, 0, sizeof(int32_t), stream) != cudaSuccess)
     return PK_ERR_CUDA;
+  TimedLaunch timed(PK_KERNEL_BWD, stream);
   kern<<<sm_count(), kBwdThreads, smem_bytes, stream>>>(
       tq, tk, tv, tdo, reinterpret_cast<const int4*>(ws + lay.off[PK_WS_BWD_ITEMS]),
       reinterpret_cast<const int32_t*>(ws + lay.off[PK_WS_BWD_ORDER]), hdr, lse,
@@ -528,6 +529,7 @@ extern "C" int pk_attn_bwd(const void* dout, const void* q, const void* k, const
     const int64_t rows = (int64_t)T * Hq;
     const int warps = 8;
     const unsigned blocks = (unsigned)((rows + warps - 1) / warps);
+    TimedLaunch timed(PK_KERNEL_DELTA, stream);
     if (out_dtype == PK_BF16)
       delta_kernel<__nv_bfloat16><<<blocks, warps * 32, 0, stream>>>(
           static_cast<const __nv_bfloat16*>(dout), static_cast<const __nv_bfloat16*>(out), delta,
@@ -569,6 +571,7 @@ extern "C" int pk_attn_bwd(const void* dout, const void* q, const void* k, const
     const int64_t n_pairs = (int64_t)T * Hq * (D / 2);
     const int threads = 256;
     const unsigned blocks = (unsigned)((n_pairs + threads - 1) / threads);
+    TimedLaunch timed(PK_KERNEL_DQ_FINISH, stream);
     if (grad_dtype == PK_BF16)
       dq_finish_kernel<__nv_bfloat16><<<blocks, threads, 0, stream>>>(
           dq_acc, static_cast<__nv_bfloat16*>(dq), reinterpret_cast<const float2*>(table), n_pairs,

@@ -306,18 +306,15 @@ int launch_fwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& 
                const WorkspaceLayout& lay, void* out, float* lse, int T, int Hq, int Hkv,
                float scale, cudaStream_t stream) {
   auto kern = attn_fwd_kernel<D, kRope, OutT>;
-  static bool configured = false;   // per template instance; attribute is per function
   const int smem_bytes = FwdSmem<D>::kDynamic;
-  if (!configured) {
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes) !=
-        cudaSuccess)
-      return PK_ERR_CUDA;
-    configured = true;
-  }
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes) !=
+      cudaSuccess)
+    return PK_ERR_CUDA;
   int32_t* hdr = reinterpret_cast<int32_t*>(ws + lay.off[PK_WS_HEADER]);
   if (cudaMemsetAsync(hdr + kHdrFwdTicket, 0, sizeof(int32_t), stream) != cudaSuccess)
     return PK_ERR_CUDA;
   const int grid = 2 * sm_count();
+  TimedLaunch timed(PK_KERNEL_FWD, stream);
   kern<<<grid, kFwdThreads, smem_bytes, stream>>>(
       tq, tk, tv, reinterpret_cast<const int4*>(ws + lay.off[PK_WS_FWD_ITEMS]),
       reinterpret_cast<const int32_t*>(ws + lay.off[PK_WS_FWD_ORDER]), hdr,
@@ -337,7 +334,7 @@ extern "C" int pk_attn_fwd(const void* q, const void* k, const void* v,
                            size_t workspace_bytes, void* stream_) {
   using namespace pk;
   cudaStream_t stream = static_cast<cudaStream_t>(stream_);
-  if (T < 0 || Hq <= 0 || Hkv <= 0) return PK_ERR_INVALID_ARG;
+  if (T < 0 || Hq <= 0 || Hkv <= 0 || !(softmax_scale > 0.f)) return PK_ERR_INVALID_ARG;
   if (!shape_supported(T, Hq, Hkv, D)) return PK_ERR_UNSUPPORTED;
   if (out_dtype != PK_BF16 && out_dtype != PK_F32) return PK_ERR_UNSUPPORTED;
   if (workspace == nullptr || (reinterpret_cast<uintptr_t>(workspace) & 255u) != 0)

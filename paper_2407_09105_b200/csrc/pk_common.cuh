@@ -80,6 +80,19 @@ __device__ inline void set_status(int32_t* header, int32_t code, int32_t detail)
 
 inline int launch_status() { return cudaGetLastError() == cudaSuccess ? PK_OK : PK_ERR_CUDA; }
 
+// Optional event pair recorded around one kernel's launches (pk_set_timing_events).
+extern cudaEvent_t g_timing_events[PK_NUM_KERNELS][2];
+struct TimedLaunch {
+  int which;
+  cudaStream_t stream;
+  TimedLaunch(int w, cudaStream_t s) : which(w), stream(s) {
+    if (g_timing_events[which][0]) cudaEventRecord(g_timing_events[which][0], stream);
+  }
+  ~TimedLaunch() {
+    if (g_timing_events[which][1]) cudaEventRecord(g_timing_events[which][1], stream);
+  }
+};
+
 // internal entry points shared between translation units
 int plan_launch(const int32_t* position_ids, int32_t T, int32_t* cu_seqlens, int32_t* n_examples,
                 int32_t* max_seqlen, void* workspace, const WorkspaceLayout& lay,

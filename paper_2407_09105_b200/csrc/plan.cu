@@ -183,6 +183,7 @@ int plan_launch(const int32_t* position_ids, int32_t T, int32_t* cu_seqlens, int
                 int32_t* max_seqlen, void* workspace, const WorkspaceLayout& lay,
                 cudaStream_t stream) {
   char* ws = static_cast<char*>(workspace);
+  TimedLaunch timed(PK_KERNEL_PLAN, stream);
   plan_kernel<<<1, kPlanThreads, 0, stream>>>(
       position_ids, T, cu_seqlens, n_examples, max_seqlen,
       reinterpret_cast<int32_t*>(ws + lay.off[PK_WS_HEADER]),
