@@ -162,6 +162,31 @@ int pk_attn_bwd(const void* dout, const void* q, const void* k, const void* v,
 int pk_status_read(const void* workspace, void* stream, int32_t* code, int32_t* detail);
 
 /*
+ * pk_seqlens_from_posids for callers that cannot give the library a workspace and for whom
+ * a device allocation is not an option (the paper has no counterpart; it is the same
+ * boundary recovery as pk_seqlens_from_posids with the same outputs).  Typical callers: a
+ * collation or data-loading thread that wants cu_seqlens for the next batch while the
+ * training framework's caching allocator already holds nearly all device memory, so that a
+ * cudaMalloc from a side library may fail; and latency-sensitive loops, because
+ * cudaMalloc/cudaFree synchronise the whole device.  This call allocates nothing and frees
+ * nothing: its scratch is a fixed array inside the library, PK_NOALLOC_MAX_TOKENS tokens
+ * large (about 1.6 MB, resident on every GPU that loads the library until the process ends).
+ *   - T > PK_NOALLOC_MAX_TOKENS returns PK_ERR_TOO_LARGE and launches nothing.
+ *   - The first call on each device looks up the array's device address (one-time set-up,
+ *     with that device current); make that first call before any stream capture begins.
+ *   - All calls on a device share the one array: two calls whose kernels can overlap on the
+ *     GPU (different streams without an ordering between them) race.  Order them.
+ *   - Only cu_seqlens, n_examples and max_seqlen are delivered; the attention calls still
+ *     take a caller workspace and plan for themselves.
+ * Arguments as for pk_seqlens_from_posids.
+ */
+#define PK_NOALLOC_MAX_TOKENS 32768
+#define PK_ERR_TOO_LARGE      8   /* size beyond a fixed built-in capacity */
+int pk_seqlens_from_posids_noalloc(const int32_t* position_ids, int32_t T,
+                                   int32_t* cu_seqlens, int32_t* n_examples,
+                                   int32_t* max_seqlen, void* stream);
+
+/*
  * Measurement aid (no counterpart in the paper): asks the library to record the CUDA
  * events `start` and `stop` (cudaEvent_t passed as void*, owned by the caller) on the
  * call's stream immediately before and after every later launch of kernel `which`

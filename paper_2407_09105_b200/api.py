@@ -20,6 +20,9 @@ PK_ERR_BAD_POSIDS = 5
 PK_ERR_TIMEOUT = 6
 PK_ERR_NO_PLAN = 7
 
+PK_ERR_TOO_LARGE = 8
+PK_NOALLOC_MAX_TOKENS = 32768
+
 PK_BF16 = 0
 PK_F32 = 1
 
@@ -46,6 +49,7 @@ _SIGNATURES = {
                                    _vp, _vp, _vp, _i32, _i32, _vp, _sz, _vp]),
     "pk_status_read": (ctypes.c_int, [_vp, _vp, ctypes.POINTER(_i32), ctypes.POINTER(_i32)]),
     "pk_set_timing_events": (ctypes.c_int, [_i32, _vp, _vp]),
+    "pk_seqlens_from_posids_noalloc": (ctypes.c_int, [_vp, _i32, _vp, _vp, _vp, _vp]),
 }
 
 EXPORTED_SYMBOLS = tuple(_SIGNATURES)
@@ -134,6 +138,21 @@ def pk_seqlens_from_posids(position_ids: torch.Tensor, cu_seqlens: torch.Tensor,
            lib().pk_seqlens_from_posids(_ptr(position_ids), T, _ptr(cu_seqlens), _ptr(n_examples),
                                         _ptr(max_seqlen), _ptr(workspace), workspace.numel(),
                                         _stream(stream)))
+
+
+def pk_seqlens_from_posids_noalloc(position_ids: torch.Tensor, cu_seqlens: torch.Tensor,
+                                   n_examples: torch.Tensor, max_seqlen: torch.Tensor,
+                                   stream=None) -> None:
+    """Boundary recovery with the library's built-in scratch: no workspace argument and no
+    allocation of any kind.  For callers that must not (or cannot) allocate device memory --
+    e.g. a collation thread running while the framework's caching allocator owns the GPU's
+    memory.  At most ``PK_NOALLOC_MAX_TOKENS`` tokens; calls on one device share the scratch,
+    so keep them ordered on the GPU."""
+    T = position_ids.numel()
+    _check("pk_seqlens_from_posids_noalloc",
+           lib().pk_seqlens_from_posids_noalloc(_ptr(position_ids), T, _ptr(cu_seqlens),
+                                                _ptr(n_examples), _ptr(max_seqlen),
+                                                _stream(stream)))
 
 
 def pk_rope_apply(x: torch.Tensor, position_ids: torch.Tensor, theta: float,

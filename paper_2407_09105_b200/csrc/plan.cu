@@ -212,3 +212,58 @@ extern "C" int pk_seqlens_from_posids(const int32_t* position_ids, int32_t T,
   return pk::plan_launch(position_ids, T, cu_seqlens, n_examples, max_seqlen, workspace, lay,
                          static_cast<cudaStream_t>(stream));
 }
+
+// ---------------------------------------------------------------------------------------
+// Boundary recovery without a caller-provided workspace and without any allocation.
+// ---------------------------------------------------------------------------------------
+namespace pk {
+namespace {
+
+// Upper bound of WorkspaceLayout::plan_total for T <= PK_NOALLOC_MAX_TOKENS: header, two
+// item lists (16 B per entry), two orders, cu_seqlens copy, per-example bases, sort cursors,
+// plus one 256-byte alignment gap per section.
+constexpr size_t kNoAllocBytes =
+    (size_t)PK_NOALLOC_MAX_TOKENS * (16 + 16 + 4 + 4 + 4 + 4) + 8 * (PK_NOALLOC_MAX_TOKENS / 128 + 4) +
+    16 + 10 * 256;
+
+// Scratch of the no-allocation entry point.  One copy lives on every GPU that loads the
+// library, from load until the process exits.  In host code this name is only a handle for
+// cudaGetSymbolAddress; kernels must be given the address that call returns.
+static __device__ __align__(256) unsigned char g_noalloc_plan_scratch[kNoAllocBytes];
+
+constexpr int kMaxDevices = 64;
+void* g_noalloc_ptr[kMaxDevices] = {};
+
+// Device address of the scratch array on the current device (looked up once per device).
+int noalloc_scratch(void** out) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return PK_ERR_CUDA;
+  if (g_noalloc_ptr[dev] == nullptr) {
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_noalloc_plan_scratch) != cudaSuccess || p == nullptr)
+      return PK_ERR_CUDA;
+    g_noalloc_ptr[dev] = p;
+  }
+  *out = g_noalloc_ptr[dev];
+  return PK_OK;
+}
+
+}  // namespace
+}  // namespace pk
+
+extern "C" int pk_seqlens_from_posids_noalloc(const int32_t* position_ids, int32_t T,
+                                              int32_t* cu_seqlens, int32_t* n_examples,
+                                              int32_t* max_seqlen, void* stream) {
+  if (T < 0 || cu_seqlens == nullptr) return PK_ERR_INVALID_ARG;
+  if (T > 0 && position_ids == nullptr) return PK_ERR_INVALID_ARG;
+  if (T > PK_NOALLOC_MAX_TOKENS) return PK_ERR_TOO_LARGE;
+  const pk::WorkspaceLayout lay = pk::workspace_layout(T, 1, 1, 64);
+  if (lay.plan_total > pk::kNoAllocBytes) return PK_ERR_TOO_LARGE;
+  void* scratch = nullptr;
+  const int rc = pk::noalloc_scratch(&scratch);
+  if (rc != PK_OK) return rc;
+  // the kernel itself clears the header and the sort cursors it reads, so stale contents
+  // of the shared array from an earlier call do not matter
+  return pk::plan_launch(position_ids, T, cu_seqlens, n_examples, max_seqlen, scratch, lay,
+                         static_cast<cudaStream_t>(stream));
+}
