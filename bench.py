@@ -189,7 +189,7 @@ def main():
         run_reference(args, w)
         return
 
-    from paper_2407_09105_b200 import api
+    from paper_2407_09105_b200 import api, replicas
 
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
@@ -253,11 +253,7 @@ def main():
     clocks = sampler.stop()
     for k in kev:
         api.pk_set_timing_events(k, None, None)
-    ms_total = e0.elapsed_time(e1)
-    t_local = torch.tensor([ms_total], dtype=torch.float64, device="cuda")
-    if dist is not None:
-        dist.all_reduce(t_local, op=dist.ReduceOp.MAX)
-    ms_step = float(t_local.item()) / args.steps
+    ms_step = replicas.max_over_ranks(e0.elapsed_time(e1), dist, "cuda") / args.steps
     fwd_ms = float(np.mean([a.elapsed_time(b) for a, b in kev[api.PK_KERNEL_FWD]]))
     bwd_ms = float(np.mean([a.elapsed_time(b) for a, b in kev[api.PK_KERNEL_BWD]]))
 
@@ -291,10 +287,7 @@ def main():
             e2e_step()
         b.record(stream)
         barrier()
-        t = torch.tensor([a.elapsed_time(b)], dtype=torch.float64, device="cuda")
-        if dist is not None:
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_e2e = float(t.item()) / n_e2e
+        ms_e2e = replicas.max_over_ranks(a.elapsed_time(b), dist, "cuda") / n_e2e
         e2e = {"value": world * flops_step / (ms_e2e * 1e-3) / 1e12, "unit": UNIT,
                "ms_per_step": ms_e2e, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
 

@@ -139,8 +139,11 @@ __device__ __forceinline__ void rope_tile_inplace_bwd(uint8_t* tile, const float
       const float4 c01 = __ldg(cs + e);
       const float2 x = __bfloat1622float2(av[e]);
       const float2 y = __bfloat1622float2(bv[e]);
-      av[e] = __floats2bfloat162_rn(x.x * c01.x - y.x * c01.y, x.y * c01.z - y.y * c01.w);
-      bv[e] = __floats2bfloat162_rn(y.x * c01.x + x.x * c01.y, y.y * c01.z + x.y * c01.w);
+      // rotated values stay fp16 (see the forward kernel)
+      reinterpret_cast<uint32_t*>(&a)[e] =
+          pack_f16x2(x.x * c01.x - y.x * c01.y, x.y * c01.z - y.y * c01.w);
+      reinterpret_cast<uint32_t*>(&b)[e] =
+          pack_f16x2(y.x * c01.x + x.x * c01.y, y.y * c01.z + x.y * c01.w);
     }
     *reinterpret_cast<uint4*>(p1) = a;
     *reinterpret_cast<uint4*>(p2) = b;
@@ -223,9 +226,13 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   const uint32_t tdK = tmem + 384;    // D cols
   const uint32_t lane_off = static_cast<uint32_t>(warp * 32) << 16;
 
-  constexpr uint32_t kIdescS = make_idesc_bf16(128, 128, 0, 0);     // K x Q^T, V x dO^T
-  constexpr uint32_t kIdescKV = make_idesc_bf16(128, D, 0, 1);      // dV, dK: B = dO / Q, MN-major
-  constexpr uint32_t kIdescDQ = make_idesc_bf16(128, D, 1, 1);      // dQ: A = dS^T as MN-major
+  constexpr uint32_t kQKFmt = kRope ? kFmtF16 : kFmtBF16;   // rotated Q, K tiles are fp16
+  constexpr uint32_t kIdescS = make_idesc(128, 128, kQKFmt, kQKFmt, 0, 0);      // K Q^T
+  constexpr uint32_t kIdescDP = make_idesc(128, 128, kFmtBF16, kFmtBF16, 0, 0);  // V dO^T
+  constexpr uint32_t kIdescDV = make_idesc(128, D, kFmtBF16, kFmtBF16, 0, 1);    // P^T dO
+  // dS^T takes the format of the tiles it is multiplied with (fp16 when they were rotated)
+  constexpr uint32_t kIdescDK = make_idesc(128, D, kQKFmt, kQKFmt, 0, 1);        // dS^T Q
+  constexpr uint32_t kIdescDQ = make_idesc(128, D, kQKFmt, kQKFmt, 1, 1);        // dS K
 
   const int G = Hq / Hkv;
   const int n_items = (hdr[PK_HDR_PLAN_T] == T) ? hdr[PK_HDR_N_ITEMS] : 0;
@@ -299,7 +306,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           for (int kk = 0; kk < D / 16; ++kk) {
             const uint32_t off = (kk / 4) * L::kBoxBytes + (kk % 4) * 32;
             mma_ss(tdP, smem_desc_sw128(sV + off, 16, 1024), smem_desc_sw128(sdO + off, 16, 1024),
-                   kIdescS, kk > 0);
+                   kIdescDP, kk > 0);
           }
           mma_commit(bar_mma);
         }
@@ -336,7 +343,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
               d1 = p1 * (__uint_as_float(dp[e + 1]) - s_delta[col]);
             }
             pp[e >> 1] = pack_bf16x2(p0, p1);
-            dd[e >> 1] = pack_bf16x2(d0, d1);
+            dd[e >> 1] = kRope ? pack_f16x2(d0, d1) : pack_bf16x2(d0, d1);
           }
           tmem_st16(tS + lane_off + c * 16, pp);
           // dS^T row `tid`, query columns [32c, 32c+32): box c/2, chunks (c%2)*4 .. +3
@@ -360,12 +367,12 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
 #pragma unroll
           for (int kk = 0; kk < kBM / 16; ++kk)
             mma_ts(tdV, tS + kk * 8, smem_desc_sw128(sdO + kk * 2048, L::kBoxBytes, 1024),
-                   kIdescKV, acc | (kk > 0));
+                   kIdescDV, acc | (kk > 0));
 #pragma unroll
           for (int kk = 0; kk < kBM / 16; ++kk) {
             const uint32_t off = (kk / 4) * L::kBoxBytes + (kk % 4) * 32;
             mma_ss(tdK, smem_desc_sw128(sdS + off, 16, 1024),
-                   smem_desc_sw128(sQ + kk * 2048, L::kBoxBytes, 1024), kIdescKV, acc | (kk > 0));
+                   smem_desc_sw128(sQ + kk * 2048, L::kBoxBytes, 1024), kIdescDK, acc | (kk > 0));
           }
 #pragma unroll
           for (int kk = 0; kk < kBN / 16; ++kk)

@@ -67,8 +67,12 @@ __device__ __forceinline__ void rope_tile_inplace(uint8_t* tile, const float2* _
       const float4 c01 = __ldg(cs + e);     // (cos0, sin0, cos1, sin1)
       const float2 x = __bfloat1622float2(av[e]);
       const float2 y = __bfloat1622float2(bv[e]);
-      av[e] = __floats2bfloat162_rn(x.x * c01.x - y.x * c01.y, x.y * c01.z - y.y * c01.w);
-      bv[e] = __floats2bfloat162_rn(y.x * c01.x + x.x * c01.y, y.y * c01.z + x.y * c01.w);
+      // the rotated values are kept as fp16 (11-bit significand): the score contraction then
+      // runs fp16 x fp16, which loses 8x less to rounding than re-rounding to bf16
+      reinterpret_cast<uint32_t*>(&a)[e] =
+          pack_f16x2(x.x * c01.x - y.x * c01.y, x.y * c01.z - y.y * c01.w);
+      reinterpret_cast<uint32_t*>(&b)[e] =
+          pack_f16x2(y.x * c01.x + x.x * c01.y, y.y * c01.z + x.y * c01.w);
     }
     *reinterpret_cast<uint4*>(p1) = a;
     *reinterpret_cast<uint4*>(p2) = b;
@@ -146,8 +150,9 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   const uint32_t tO = tmem + 128;      // D fp32 columns
   const uint32_t lane_off = static_cast<uint32_t>(warp * 32) << 16;
 
-  constexpr uint32_t kIdescQK = make_idesc_bf16(128, 128, 0, 0);
-  constexpr uint32_t kIdescPV = make_idesc_bf16(128, D, 0, 1);
+  constexpr uint32_t kQKFmt = kRope ? kFmtF16 : kFmtBF16;   // rotated tiles are fp16
+  constexpr uint32_t kIdescQK = make_idesc(128, 128, kQKFmt, kQKFmt, 0, 0);
+  constexpr uint32_t kIdescPV = make_idesc(128, D, kFmtBF16, kFmtBF16, 0, 1);
 
   const int G = Hq / Hkv;
   const int n_items = (hdr[PK_HDR_PLAN_T] == T) ? hdr[PK_HDR_N_ITEMS] : 0;

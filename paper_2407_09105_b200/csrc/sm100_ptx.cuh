@@ -163,11 +163,15 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr, uint32_t lbo
   return d;
 }
 
-// Instruction descriptor: bf16 x bf16 -> fp32, dense.
-__host__ __device__ constexpr uint32_t make_idesc_bf16(int M, int N, int a_mn_major, int b_mn_major) {
+// Instruction descriptor of kind::f16: 16-bit A and B, fp32 accumulator, dense.  A and B
+// must have the SAME format (both fp16 or both bf16): a mixed pair is rejected by the
+// hardware as an illegal instruction.
+constexpr uint32_t kFmtF16 = 0, kFmtBF16 = 1;
+__host__ __device__ constexpr uint32_t make_idesc(int M, int N, uint32_t a_fmt, uint32_t b_fmt,
+                                                  int a_mn_major, int b_mn_major) {
   return (1u << 4)                      // accumulator fp32
-         | (1u << 7)                    // A bf16
-         | (1u << 10)                   // B bf16
+         | (a_fmt << 7)
+         | (b_fmt << 10)
          | ((uint32_t)a_mn_major << 15)
          | ((uint32_t)b_mn_major << 16)
          | ((uint32_t)(N >> 3) << 17)
@@ -204,6 +208,11 @@ __device__ __forceinline__ float fast_exp2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
+}
+__device__ __forceinline__ uint32_t pack_f16x2(float lo, float hi) {
+  uint32_t r;
+  asm("cvt.rn.satfinite.f16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+  return r;
 }
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   uint32_t r;

@@ -1,0 +1,115 @@
+"""Parity on the five configurations.  c1 and c2 are checked in full against the oracle;
+c3, c4, c5 run at full size in the launch configuration the benchmark times (one flat stream,
+bf16 outputs) and are checked on whole sampled examples plus single rows the oracle computes
+one by one (any row of O / lse / dQ is cheap; dK / dV need whole examples).
+Tolerances as in the other parity tests: 1e-2 (O, lse), 2e-2 (grads), plus half a bf16 ulp of
+the exact value for bf16 outputs."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import packed_attention as orc
+from paper_2407_09105_b200 import api, workloads as wl
+from helpers import f64, max_abs, run_bwd, run_fwd, to_cuda
+
+pytestmark = pytest.mark.gpu
+
+
+def _close(g, e, tol, bf16):
+    g, e = np.asarray(g), np.asarray(e)
+    lim = tol + (2.0 ** -8 * np.abs(e) if bf16 else 0.0)
+    return bool((np.abs(g - e) <= lim).all())
+
+
+def test_c1_full_fp32_and_bf16():
+    w = wl.workload("c1")
+    st = to_cuda(wl.stream_tensors(w, w.streams[0], 0))
+    pos = st.position_ids.cpu().numpy()
+    eo, el = orc.attn_fwd(f64(st.q), f64(st.k), f64(st.v), pos, w.softmax_scale)
+    eg = orc.attn_bwd(f64(st.dout), f64(st.q), f64(st.k), f64(st.v), pos, w.softmax_scale)
+    for dt in (torch.float32, torch.bfloat16):
+        out, lse, ws = run_fwd(st, w, dt)
+        gr = run_bwd(st, w, out, lse, ws, dt)
+        bf = dt == torch.bfloat16
+        assert _close(f64(out), eo, 1e-2, bf) and _close(f64(lse), el, 1e-2, False)
+        for g, e in zip(gr, eg):
+            assert _close(f64(g), e, 2e-2, bf)
+
+
+def test_c2_full_flat_stream_fp32():
+    w = wl.workload("c2")
+    lens = w.flat_lengths()
+    st = to_cuda(wl.stream_tensors(w, lens, 0))
+    out, lse, ws = run_fwd(st, w, torch.float32)
+    dq, dk, dv = run_bwd(st, w, out, lse, ws, torch.float32)
+    pos = st.position_ids.cpu().numpy()
+    q, k, v, do = (f64(x) for x in (st.q, st.k, st.v, st.dout))
+    eo, el = orc.attn_fwd(q, k, v, pos, w.softmax_scale, w.rope_theta)
+    assert max_abs(f64(out), eo) <= 1e-2 and max_abs(f64(lse), el) <= 1e-2
+    edq, edk, edv = orc.attn_bwd(do, q, k, v, pos, w.softmax_scale, w.rope_theta)
+    assert max_abs(f64(dq), edq) <= 2e-2
+    assert max_abs(f64(dk), edk) <= 2e-2
+    assert max_abs(f64(dv), edv) <= 2e-2
+
+
+def _sampled(name, n_rows=48, max_example=2600):
+    w = wl.workload(name)
+    lens = w.flat_lengths()
+    st = wl.stream_tensors(w, lens, 0, device="cuda")
+    T, Hq, D = st.q.shape
+    out, lse, ws = run_fwd(st, w, torch.bfloat16)
+    dq, dk, dv = run_bwd(st, w, out, lse, ws, torch.bfloat16)
+    pos = st.position_ids.cpu().numpy()
+    cu, E, _ = orc.seqlens_from_posids(pos)
+    rng = np.random.default_rng(7)
+
+    # (a) whole examples: the shortest, those next to a multiple of 128, first and last, a few random
+    L = np.diff(cu[:E + 1])
+    cand = {0, E - 1, int(np.argmin(L))}
+    cand |= {int(e) for e in np.flatnonzero((L % 128 <= 1) | (L % 128 == 127))[:3]}
+    cand |= {int(e) for e in rng.choice(E, size=min(4, E), replace=False)}
+    mid = [int(e) for e in np.argsort(L) if L[e] <= max_example]
+    cand.add(mid[-1])                                     # the longest affordable example
+    cand = sorted(e for e in cand if L[e] <= max_example)
+    for e in cand:
+        s, t = int(cu[e]), int(cu[e + 1])
+        sl = slice(s, t)
+        q, k, v, do = (f64(x[sl]) for x in (st.q, st.k, st.v, st.dout))
+        eo, el = orc.attn_fwd(q, k, v, pos[sl], w.softmax_scale, w.rope_theta)
+        assert _close(f64(out[sl]), eo, 1e-2, True), (name, e)
+        assert _close(f64(lse[:, sl]), el, 1e-2, False), (name, e)
+        edq, edk, edv = orc.attn_bwd(do, q, k, v, pos[sl], w.softmax_scale, w.rope_theta)
+        assert _close(f64(dq[sl]), edq, 2e-2, True), (name, e, "dq")
+        assert _close(f64(dk[sl]), edk, 2e-2, True), (name, e, "dk")
+        assert _close(f64(dv[sl]), edv, 2e-2, True), (name, e, "dv")
+
+    # (b) single rows anywhere, including the last row of the longest example
+    e_long = int(np.argmax(L))
+    rows = [int(cu[e_long + 1]) - 1, int(cu[e_long]) + int(L[e_long]) // 2]
+    rows += [int(x) for x in rng.integers(0, T, size=n_rows)]
+    for i in rows:
+        h = int(rng.integers(0, Hq))
+        e = int(np.searchsorted(cu[:E + 1], i, side="right") - 1)
+        s = int(cu[e])
+        sl = slice(s, i + 1)
+        qh, kh, vh, doh = (f64(x[sl]) for x in (st.q, st.k, st.v, st.dout))
+        eo, el = orc.attn_fwd_row(qh, kh, vh, pos[sl], w.softmax_scale, w.rope_theta, i - s, h)
+        assert _close(f64(out[i, h]), eo, 1e-2, True), (name, i, h)
+        assert abs(float(lse[h, i]) - el) <= 1e-2, (name, i, h)
+        edq = orc.attn_bwd_dq_row(doh, qh, kh, vh, pos[sl], w.softmax_scale, w.rope_theta, i - s, h)
+        assert _close(f64(dq[i, h]), edq, 2e-2, True), (name, i, h, "dq")
+    # no row of any output was left unwritten
+    for x in (out, lse, dq, dk, dv):
+        assert not torch.isnan(x).any()
+
+
+def test_c3_sampled_full_size():
+    _sampled("c3")
+
+
+def test_c4_sampled_full_size():
+    _sampled("c4")
+
+
+def test_c5_sampled_full_size():
+    _sampled("c5", n_rows=24, max_example=9000)
