@@ -179,12 +179,17 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--workload", default="c4")
     ap.add_argument("--impl", default="ours")
+    ap.add_argument("--packs", type=int, default=0,
+                    help="use only the first N packs of the workload (small cases for profiling)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl != "reference" else args.warmup
 
     w = wl.workload(args.workload)
+    if args.packs > 0:
+        w = wl.Workload(f"{w.name}[:{args.packs}]", w.seed, w.num_q_heads, w.num_kv_heads,
+                        w.head_dim, w.rope_theta, w.streams[:args.packs], w.packing)
     if args.impl == "reference":
         run_reference(args, w)
         return
