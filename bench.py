@@ -239,7 +239,8 @@ def main():
 
     # per-kernel events: recorded by the library around the two main kernels
     kev = {k: [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
-               for _ in range(args.steps)] for k in (api.PK_KERNEL_FWD, api.PK_KERNEL_BWD)}
+               for _ in range(args.steps)]
+           for k in (api.PK_KERNEL_FWD, api.PK_KERNEL_BWD, api.PK_KERNEL_BWD_DQ)}
     for pairs in kev.values():
         for a, b in pairs:
             a.record(stream)
@@ -261,6 +262,7 @@ def main():
     ms_step = replicas.max_over_ranks(e0.elapsed_time(e1), dist, "cuda") / args.steps
     fwd_ms = float(np.mean([a.elapsed_time(b) for a, b in kev[api.PK_KERNEL_FWD]]))
     bwd_ms = float(np.mean([a.elapsed_time(b) for a, b in kev[api.PK_KERNEL_BWD]]))
+    dq_ms = float(np.mean([a.elapsed_time(b) for a, b in kev[api.PK_KERNEL_BWD_DQ]])) if theta <= 0 else 0.0
 
     flops_step = w.useful_flops_fwd + w.useful_flops_bwd
     value = world * flops_step / (ms_step * 1e-3) / 1e12
@@ -302,7 +304,13 @@ def main():
         return
 
     peaks = _peaks()
-    bwd_tflops = w.useful_flops_bwd / (bwd_ms * 1e-3) / 1e12
+    # without fused RoPE the backward is two kernels: dK/dV (6 of the 10 useful FLOPs per pair and
+    # head-dim: dV, dK, plus one of the two recomputed products) and dQ.  The dominant kernel is
+    # the dK/dV one; its useful work is dV and dK only: 4*D FLOPs per pair.
+    split = theta <= 0
+    bwd_flops = (w.useful_flops_bwd * 4 // 10) if split else w.useful_flops_bwd
+    bwd_tflops = bwd_flops / (bwd_ms * 1e-3) / 1e12
+    executed = ((8 if split else 10) * D * Hq * w.causal_pairs) / (bwd_ms * 1e-3) / 1e12
     fwd_tflops = w.useful_flops_fwd / (fwd_ms * 1e-3) / 1e12
     roofline = {
         "kernel": "attn_bwd_kernel", "bound": "tensor", "achieved": bwd_tflops,
@@ -311,6 +319,12 @@ def main():
         "traffic": (None if NCU_BWD_DRAM_BYTES_PER_PAIR is None
                     else NCU_BWD_DRAM_BYTES_PER_PAIR * w.causal_pairs * Hq),
         "ms_per_launch": bwd_ms,
+        "note": ("dK/dV kernel: useful = dV and dK (4*D FLOPs per causal pair and head); it also "
+                 "recomputes S and dP, executed_tflops counts those" if split else "fused-RoPE kernel"),
+        "executed_tflops": executed,
+        "bwd_dq_kernel": ({"achieved": (w.useful_flops_bwd * 2 // 10) / (dq_ms * 1e-3) / 1e12,
+                           "executed_tflops": (6 * D * Hq * w.causal_pairs) / (dq_ms * 1e-3) / 1e12,
+                           "ms_per_launch": dq_ms} if split else None),
         "fwd_kernel": {"achieved": fwd_tflops, "frac": fwd_tflops / peaks["sustained"],
                        "ms_per_launch": fwd_ms},
     }
@@ -333,7 +347,7 @@ def main():
         "pct_of_bf16_peak": {"sustained": 100 * value / world / peaks["sustained"],
                              "burst": 100 * value / world / peaks["burst"],
                              "source": peaks["source"]},
-        "clocks": clocks, "e2e": e2e, "gpu_launches": 5 * args.steps + (2 * args.steps if theta > 0 else 0),
+        "clocks": clocks, "e2e": e2e, "gpu_launches": (5 + (2 if theta > 0 else 0)) * args.steps,
         "roofline": roofline, "cpu_baseline": cpu_baseline,
     }
     print(json.dumps(line))

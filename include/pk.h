@@ -196,9 +196,10 @@ int pk_seqlens_from_posids_noalloc(const int32_t* position_ids, int32_t T,
 #define PK_KERNEL_PLAN      0
 #define PK_KERNEL_FWD       1
 #define PK_KERNEL_DELTA     2
-#define PK_KERNEL_BWD       3
+#define PK_KERNEL_BWD       3   /* dK/dV kernel (the whole backward when RoPE is fused) */
 #define PK_KERNEL_DQ_FINISH 4
-#define PK_NUM_KERNELS      5
+#define PK_KERNEL_BWD_DQ    5   /* dQ kernel */
+#define PK_NUM_KERNELS      6
 int pk_set_timing_events(int32_t which, void* start, void* stop);
 
 #ifdef __cplusplus

@@ -196,7 +196,7 @@ def pk_status_read(workspace: torch.Tensor, stream=None) -> Tuple[int, int]:
     return code.value, detail.value
 
 
-PK_KERNEL_PLAN, PK_KERNEL_FWD, PK_KERNEL_DELTA, PK_KERNEL_BWD, PK_KERNEL_DQ_FINISH = range(5)
+PK_KERNEL_PLAN, PK_KERNEL_FWD, PK_KERNEL_DELTA, PK_KERNEL_BWD, PK_KERNEL_DQ_FINISH, PK_KERNEL_BWD_DQ = range(6)
 
 
 def pk_set_timing_events(which: int, start: Optional[torch.cuda.Event],

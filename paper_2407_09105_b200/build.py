@@ -13,7 +13,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libpk.so")
-SOURCES = ["api.cu", "plan.cu", "rope.cu", "attn_fwd.cu", "attn_bwd.cu"]
+SOURCES = ["api.cu", "plan.cu", "rope.cu", "attn_fwd.cu", "attn_bwd.cu", "attn_bwd_ws.cu"]
 
 
 def _nvcc() -> str:
@@ -40,6 +40,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
            "-shared", "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", CSRC]
     if verbose:
         cmd += ["-Xptxas", "-v"]
+    cmd += os.environ.get("PK_NVCC_EXTRA", "").split()
     cmd += srcs + ["-o", LIB]
     res = subprocess.run(cmd, capture_output=True, text=True)
     if verbose or res.returncode != 0:

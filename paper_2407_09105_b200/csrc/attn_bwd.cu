@@ -16,6 +16,7 @@
 //                                           for dK and MN-major for dQ)
 #include <cuda_bf16.h>
 
+#include "attn_common.cuh"
 #include "pk_common.cuh"
 #include "sm100_ptx.cuh"
 #include "tensor_map.cuh"
@@ -147,32 +148,6 @@ __device__ __forceinline__ void rope_tile_inplace_bwd(uint8_t* tile, const float
     }
     *reinterpret_cast<uint4*>(p1) = a;
     *reinterpret_cast<uint4*>(p2) = b;
-  }
-}
-
-__device__ __forceinline__ void red_add_v4(float* addr, float a, float b, float c, float d) {
-  asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};"
-               ::"l"(addr), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
-}
-
-template <typename GradT>
-__device__ __forceinline__ void store_chunk32(GradT* dst, const float* x);
-template <>
-__device__ __forceinline__ void store_chunk32<float>(float* dst, const float* x) {
-#pragma unroll
-  for (int c = 0; c < 32; c += 4)
-    *reinterpret_cast<float4*>(dst + c) = make_float4(x[c], x[c + 1], x[c + 2], x[c + 3]);
-}
-template <>
-__device__ __forceinline__ void store_chunk32<__nv_bfloat16>(__nv_bfloat16* dst, const float* x) {
-#pragma unroll
-  for (int c = 0; c < 32; c += 8) {
-    uint4 o;
-    o.x = pack_bf16x2(x[c], x[c + 1]);
-    o.y = pack_bf16x2(x[c + 2], x[c + 3]);
-    o.z = pack_bf16x2(x[c + 4], x[c + 5]);
-    o.w = pack_bf16x2(x[c + 6], x[c + 7]);
-    *reinterpret_cast<uint4*>(dst + c) = o;
   }
 }
 
@@ -545,7 +520,9 @@ extern "C" int pk_attn_bwd(const void* dout, const void* q, const void* k, const
       delta_kernel<float><<<blocks, warps * 32, 0, stream>>>(
           static_cast<const __nv_bfloat16*>(dout), static_cast<const float*>(out), delta, T, Hq, D);
     if ((rc = launch_status()) != PK_OK) return rc;
-    if (cudaMemsetAsync(dq_acc, 0, sizeof(float) * (size_t)T * Hq * D, stream) != cudaSuccess)
+    // only the fused-RoPE kernel accumulates dQ with reductions and needs a cleared buffer
+    if (use_rope &&
+        cudaMemsetAsync(dq_acc, 0, sizeof(float) * (size_t)T * Hq * D, stream) != cudaSuccess)
       return PK_ERR_CUDA;
   }
 
@@ -554,6 +531,11 @@ extern "C" int pk_attn_bwd(const void* dout, const void* q, const void* k, const
   if (!make_tile_map_bf16(&tq, q, T, Hq * D) || !make_tile_map_bf16(&tk, k, T, Hkv * D) ||
       !make_tile_map_bf16(&tv, v, T, Hkv * D) || !make_tile_map_bf16(&tdo, dout, T, Hq * D))
     return PK_ERR_CUDA;
+  if (!use_rope) {
+    // two warp-specialised kernels (dK/dV, then dQ); dQ is final, no finishing pass
+    return launch_bwd_ws(tq, tk, tv, tdo, ws, lay, lse, dq, dk, dv, T, Hq, Hkv, D, grad_dtype,
+                         softmax_scale, stream);
+  } else {
 #define PK_BWD(DD, RR, TT)                                                                      \
   rc = launch_bwd<DD, RR, TT>(tq, tk, tv, tdo, ws, lay, lse, dk, dv, T, Hq, Hkv, softmax_scale, \
                               stream)
@@ -571,6 +553,7 @@ extern "C" int pk_attn_bwd(const void* dout, const void* q, const void* k, const
     }
   }
 #undef PK_BWD
+  }
   if (rc != PK_OK) return rc;
 
   // (3) dQ: scale, rotate back, cast

@@ -1,0 +1,692 @@
+// Warp-specialised backward kernels (no fused RoPE) for sm_100a.
+//
+// The backward is split into two kernels so that no gradient needs floating-point atomics
+// (fp32 reductions into a dQ accumulator ran at about 2 TB/s here and took longer than all
+// the tensor-core work together; a TMA reduce-add reached 2.7 TB/s, still not enough):
+//
+//   attn_bwd_dkv_kernel  key-block stationary, unit = (<=128 key rows of one example, kv head):
+//       for each of the G query heads and each query tile from the diagonal to the example end
+//         S^T = K Q^T, dP^T = V dO^T, P^T = exp2(..), dS^T = P^T o (dP^T - delta),
+//         dV += P^T dO, dK += dS^T Q            (dK, dV stay in tensor memory for the unit)
+//   attn_bwd_dq_kernel   query-block stationary, unit = (<=128 query rows of one example, q head):
+//       for each key tile from the example start to the diagonal
+//         S = Q K^T, dP = dO V^T, dS = P o (dP - delta), dQ += dS K   (dQ stays in tensor memory)
+//
+// Both recompute S and dP (7 contractions per tile pair instead of 5), both are bitwise
+// reproducible, and both never visit a tile outside an example's causal block.
+//
+// Roles (320 threads): warps 0-7 compute (lane = tensor-memory row; warps 0-3 take columns
+// 0..63, warps 4-7 columns 64..127), warp 8 issues every tcgen05.mma, warp 9 drives TMA.
+// Units are assigned statically: CTA c takes positions c, 2P-1-c, 2P+c, ... of the plan's
+// longest-first order, so the roles enumerate the same sequence without talking to each other.
+// Every wait is bounded; on expiry an abort flag makes all later waits return at once.
+#include <cuda_bf16.h>
+
+#include "attn_common.cuh"
+#include "pk_common.cuh"
+#include "sm100_ptx.cuh"
+#include "tensor_map.cuh"
+
+namespace pk {
+namespace {
+
+using namespace ptx;
+
+constexpr int kWsThreads = 320;
+constexpr int kComputeThreads = 256;
+constexpr int kMmaWarp = 8;
+constexpr int kLoadWarp = 9;
+constexpr float kLog2eWs = 1.4426950408889634f;
+
+// position in the longest-first order of the r-th unit of this CTA (snake over the rounds)
+__device__ __forceinline__ int snake_unit(int r, int cta, int n_cta) {
+  return r * n_cta + ((r & 1) ? (n_cta - 1 - cta) : cta);
+}
+__device__ __forceinline__ void compute_bar_sync() {
+  asm volatile("bar.sync 1, 256;" ::: "memory");
+}
+
+// =========================================================================================
+// dK / dV kernel
+// =========================================================================================
+template <int D>
+struct DkvSmem {
+  static constexpr int kBoxBytes = 128 * 128;
+  static constexpr int kBoxes = D / 64;
+  static constexpr int kTileBytes = kBoxBytes * kBoxes;
+  static constexpr int kK = 0;
+  static constexpr int kV = kTileBytes;
+  static constexpr int kQ0 = 2 * kTileBytes;                 // stage s: Q at kQ0 + s*2*tile
+  static constexpr int kStageBytes = 2 * kTileBytes;         // Q then dO
+  static constexpr int kdS = kQ0 + 2 * kStageBytes;          // 2 boxes
+  static constexpr int kLse = kdS + 2 * kBoxBytes;           // [2][128] floats
+  static constexpr int kDelta = kLse + 1024;                 // [2][128] floats
+  static constexpr int kBars = kDelta + 1024;
+  static constexpr int kMisc = kBars + 16 * 8;
+  static constexpr int kTotal = kMisc + 16;
+};
+
+enum DkvBar {
+  kvKvFull = 0, kvKvEmpty, kvQFull0, kvQFull1, kvDoFull0, kvDoFull1, kvQdoEmpty0, kvQdoEmpty1,
+  kvSFull, kvDpFull, kvPReady, kvDsReady, kvUnitDone, kvDkvRead, kvNumBars
+};
+
+template <int D, typename GradT>
+__global__ void __launch_bounds__(kWsThreads, 1)
+attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+                    const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_do,
+                    const int4* __restrict__ items, const int32_t* __restrict__ order, int32_t* hdr,
+                    const float* __restrict__ lse, const float* __restrict__ delta,
+                    GradT* __restrict__ dk, GradT* __restrict__ dv,
+                    int T, int Hq, int Hkv, float scale, float scale_log2) {
+  using L = DkvSmem<D>;
+  extern __shared__ __align__(1024) uint8_t smem[];
+  const uint32_t sbase = smem_u32(smem);
+  const uint32_t sK = sbase + L::kK, sV = sbase + L::kV, sdS = sbase + L::kdS;
+  float* s_lse = reinterpret_cast<float*>(smem + L::kLse);
+  float* s_delta = reinterpret_cast<float*>(smem + L::kDelta);
+  const uint32_t bars = sbase + L::kBars;
+  auto bar = [&](int i) { return bars + 8u * (uint32_t)i; };
+  volatile int* s_tmem = reinterpret_cast<volatile int*>(smem + L::kMisc);
+  volatile int* s_abort = s_tmem + 1;
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+
+  if (tid == 0) {
+    mbar_init(bar(kvKvFull), 1);
+    mbar_init(bar(kvKvEmpty), 1);
+    mbar_init(bar(kvQFull0), 33);
+    mbar_init(bar(kvQFull1), 33);
+    mbar_init(bar(kvDoFull0), 1);
+    mbar_init(bar(kvDoFull1), 1);
+    mbar_init(bar(kvQdoEmpty0), 1);
+    mbar_init(bar(kvQdoEmpty1), 1);
+    mbar_init(bar(kvSFull), 1);
+    mbar_init(bar(kvDpFull), 1);
+    mbar_init(bar(kvPReady), kComputeThreads);
+    mbar_init(bar(kvDsReady), kComputeThreads);
+    mbar_init(bar(kvUnitDone), 1);
+    mbar_init(bar(kvDkvRead), kComputeThreads);
+    fence_mbar_init();
+    *s_abort = ((sbase & 1023u) != 0) ? 1 : 0;   // swizzled tiles need a 1024-byte aligned base
+  }
+  if (warp == kMmaWarp) {
+    tmem_alloc(smem_u32(const_cast<int*>(s_tmem)), 512);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = static_cast<uint32_t>(*s_tmem);
+  const uint32_t tS = tmem, tdP = tmem + 128, tdV = tmem + 256, tdK = tmem + 384;
+
+  const int G = Hq / Hkv;
+  const bool plan_ok = (hdr[PK_HDR_PLAN_T] == T);
+  if (!plan_ok && blockIdx.x == 0 && tid == 0) set_status(hdr, PK_ERR_NO_PLAN, T);
+  const int n_units = plan_ok ? hdr[PK_HDR_N_ITEMS] * Hkv : 0;
+  const int n_cta = gridDim.x, cta = blockIdx.x;
+
+  if (warp == kLoadWarp) {
+    // =============================== loader ===============================================
+    if (lane == 0) {
+      prefetch_tensormap(&tm_q);
+      prefetch_tensormap(&tm_k);
+      prefetch_tensormap(&tm_v);
+      prefetch_tensormap(&tm_do);
+    }
+    int gs = 0, uc = 0;
+    for (int r = 0;; ++r, ++uc) {
+      const int u = snake_unit(r, cta, n_cta);
+      if (u >= n_units || *s_abort) break;
+      const int4 it = items[order[u / Hkv]];
+      const int g = u % Hkv;
+      const int kv_start = it.x, q_start = it.z, q_len = it.w;
+      const int n_q = (q_len + kBM - 1) / kBM;
+      mbar_wait(bar(kvKvEmpty), (uc & 1) ^ 1, s_abort);
+      if (lane == 0) {
+        mbar_expect_tx(bar(kvKvFull), 2 * L::kTileBytes);
+#pragma unroll
+        for (int b = 0; b < L::kBoxes; ++b) {
+          tma_load_2d(sK + b * L::kBoxBytes, &tm_k, g * D + b * 64, kv_start, bar(kvKvFull));
+          tma_load_2d(sV + b * L::kBoxBytes, &tm_v, g * D + b * 64, kv_start, bar(kvKvFull));
+        }
+      }
+      for (int hh = 0; hh < G; ++hh) {
+        const int h = g * G + hh;
+        for (int i = 0; i < n_q; ++i, ++gs) {
+          const int st = gs & 1;
+          const int q0 = q_start + i * kBM;
+          mbar_wait(bar(kvQdoEmpty0 + st), ((gs >> 1) & 1) ^ 1, s_abort);
+          const uint32_t sQ = sbase + L::kQ0 + st * L::kStageBytes, sdO = sQ + L::kTileBytes;
+          if (lane == 0) {
+            mbar_expect_tx(bar(kvQFull0 + st), L::kTileBytes);
+#pragma unroll
+            for (int b = 0; b < L::kBoxes; ++b)
+              tma_load_2d(sQ + b * L::kBoxBytes, &tm_q, h * D + b * 64, q0, bar(kvQFull0 + st));
+            mbar_expect_tx(bar(kvDoFull0 + st), L::kTileBytes);
+#pragma unroll
+            for (int b = 0; b < L::kBoxes; ++b)
+              tma_load_2d(sdO + b * L::kBoxBytes, &tm_do, h * D + b * 64, q0, bar(kvDoFull0 + st));
+          }
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const int row = lane * 4 + e, tok = q0 + row;
+            const bool in = tok < T;
+            s_lse[st * 128 + row] = in ? lse[(size_t)h * T + tok] * kLog2eWs : 0.f;
+            s_delta[st * 128 + row] = in ? delta[(size_t)h * T + tok] : 0.f;
+          }
+          mbar_arrive(bar(kvQFull0 + st));
+        }
+      }
+    }
+  } else if (warp == kMmaWarp) {
+    // =============================== MMA issuer ===========================================
+    if (lane == 0) {
+      constexpr uint32_t kIdescS = make_idesc(128, 128, kFmtBF16, kFmtBF16, 0, 0);
+      constexpr uint32_t kIdescKV = make_idesc(128, D, kFmtBF16, kFmtBF16, 0, 1);
+      int gs = 0, uc = 0;
+      auto issue_s = [&](int st) {
+        const uint32_t sQ = sbase + L::kQ0 + st * L::kStageBytes;
+#pragma unroll
+        for (int kk = 0; kk < D / 16; ++kk) {
+          const uint32_t off = (kk / 4) * L::kBoxBytes + (kk % 4) * 32;
+          mma_ss(tS, smem_desc_sw128(sK + off, 16, 1024), smem_desc_sw128(sQ + off, 16, 1024),
+                 kIdescS, kk > 0);
+        }
+        mma_commit(bar(kvSFull));
+      };
+      auto issue_dp = [&](int st) {
+        const uint32_t sdO = sbase + L::kQ0 + st * L::kStageBytes + L::kTileBytes;
+#pragma unroll
+        for (int kk = 0; kk < D / 16; ++kk) {
+          const uint32_t off = (kk / 4) * L::kBoxBytes + (kk % 4) * 32;
+          mma_ss(tdP, smem_desc_sw128(sV + off, 16, 1024), smem_desc_sw128(sdO + off, 16, 1024),
+                 kIdescS, kk > 0);
+        }
+        mma_commit(bar(kvDpFull));
+      };
+      for (int r = 0;; ++r, ++uc) {
+        const int u = snake_unit(r, cta, n_cta);
+        if (u >= n_units || *s_abort) break;
+        const int4 it = items[order[u / Hkv]];
+        const int n_q = (it.w + kBM - 1) / kBM;
+        const int n_steps = G * n_q;
+        mbar_wait(bar(kvKvFull), uc & 1, s_abort);
+        // prologue: S(0), dP(0).  The compute warps finished reading S and dP of the previous
+        // unit's last step before they signalled its dS, which the last dK waited for.
+        mbar_wait(bar(kvQFull0 + (gs & 1)), (gs >> 1) & 1, s_abort);
+        tc_fence_after();
+        issue_s(gs & 1);
+        mbar_wait(bar(kvDoFull0 + (gs & 1)), (gs >> 1) & 1, s_abort);
+        tc_fence_after();
+        issue_dp(gs & 1);
+        for (int s = 0; s < n_steps; ++s, ++gs) {
+          const int st = gs & 1;
+          const uint32_t sQ = sbase + L::kQ0 + st * L::kStageBytes, sdO = sQ + L::kTileBytes;
+          const uint32_t acc = s > 0 ? 1u : 0u;
+          mbar_wait(bar(kvPReady), gs & 1, s_abort);
+          if (s == 0 && uc > 0) mbar_wait(bar(kvDkvRead), (uc - 1) & 1, s_abort);
+          tc_fence_after();
+#pragma unroll
+          for (int kk = 0; kk < kBM / 16; ++kk)   // dV += P^T dO
+            mma_ts(tdV, tS + kk * 8, smem_desc_sw128(sdO + kk * 2048, L::kBoxBytes, 1024), kIdescKV,
+                   acc | (kk > 0));
+          const bool more = (s + 1 < n_steps);
+          const int g1 = gs + 1;
+          if (more) {                              // S(s+1): P(s) was consumed by dV(s) above
+            mbar_wait(bar(kvQFull0 + (g1 & 1)), (g1 >> 1) & 1, s_abort);
+            tc_fence_after();
+            issue_s(g1 & 1);
+          }
+          mbar_wait(bar(kvDsReady), gs & 1, s_abort);
+          tc_fence_after();
+#pragma unroll
+          for (int kk = 0; kk < kBM / 16; ++kk) {   // dK += dS^T Q
+            const uint32_t off = (kk / 4) * L::kBoxBytes + (kk % 4) * 32;
+            mma_ss(tdK, smem_desc_sw128(sdS + off, 16, 1024),
+                   smem_desc_sw128(sQ + kk * 2048, L::kBoxBytes, 1024), kIdescKV, acc | (kk > 0));
+          }
+          mma_commit(bar(kvQdoEmpty0 + st));
+          if (more) {                              // dP(s+1): dP(s) was read before dS(s) was signalled
+            mbar_wait(bar(kvDoFull0 + (g1 & 1)), (g1 >> 1) & 1, s_abort);
+            tc_fence_after();
+            issue_dp(g1 & 1);
+          }
+        }
+        mma_commit(bar(kvUnitDone));
+        mma_commit(bar(kvKvEmpty));
+      }
+    }
+    __syncwarp();
+  } else {
+    // =============================== compute (warps 0-7) ==================================
+    const int row = tid & 127;              // key row inside the block
+    const int hf = tid >> 7;                // which half of the query columns
+    const uint32_t lane_off = static_cast<uint32_t>((warp & 3) * 32) << 16;
+    int gs = 0, uc = 0;
+    for (int r = 0;; ++r, ++uc) {
+      const int u = snake_unit(r, cta, n_cta);
+      if (u >= n_units || *s_abort) break;
+      const int4 it = items[order[u / Hkv]];
+      const int g = u % Hkv;
+      const int kv_start = it.x, kv_len = it.y, q_len = it.w;
+      const int n_q = (q_len + kBM - 1) / kBM;
+      for (int hh = 0; hh < G; ++hh) {
+        for (int i = 0; i < n_q; ++i, ++gs) {
+          const int st = gs & 1;
+          const int q_left = q_len - i * kBM;
+          const int col_min = (i == 0) ? row : 0;
+          const float* lse2 = s_lse + st * 128 + hf * 64;
+          const float* dl = s_delta + st * 128 + hf * 64;
+          mbar_wait(bar(kvQFull0 + st), (gs >> 1) & 1, s_abort);   // lse / delta rows visible
+          mbar_wait(bar(kvSFull), gs & 1, s_abort);
+          tc_fence_after();
+          float p[64];
+          {
+            uint32_t s0[32], s1[32];
+            tmem_ld32(tS + lane_off + hf * 64, s0);
+            tmem_ld32(tS + lane_off + hf * 64 + 32, s1);
+            tmem_wait_ld();
+#pragma unroll
+            for (int c = 0; c < 32; ++c) {
+              const int col = hf * 64 + c;
+              const bool ok = (col >= col_min) && (col < q_left);
+              const float x = fast_exp2(fmaf(__uint_as_float(s0[c]), scale_log2, -lse2[c]));
+              p[c] = ok ? x : 0.f;
+            }
+#pragma unroll
+            for (int c = 0; c < 32; ++c) {
+              const int col = hf * 64 + 32 + c;
+              const bool ok = (col >= col_min) && (col < q_left);
+              const float x = fast_exp2(fmaf(__uint_as_float(s1[c]), scale_log2, -lse2[32 + c]));
+              p[32 + c] = ok ? x : 0.f;
+            }
+          }
+          // both halves must have read S before P overwrites its columns
+          tc_fence_before();
+          compute_bar_sync();
+          tc_fence_after();
+          {
+            uint32_t pp[32];
+#pragma unroll
+            for (int c = 0; c < 32; ++c) pp[c] = pack_bf16x2(p[2 * c], p[2 * c + 1]);
+            tmem_st32(tS + lane_off + hf * 32, pp);
+            tmem_wait_st();
+          }
+          tc_fence_before();
+          mbar_arrive(bar(kvPReady));
+
+          mbar_wait(bar(kvDpFull), gs & 1, s_abort);
+          tc_fence_after();
+          uint8_t* ds_row = smem + L::kdS + hf * L::kBoxBytes + row * 128;
+#pragma unroll
+          for (int c2 = 0; c2 < 2; ++c2) {
+            uint32_t dp[32], dd[16];
+            tmem_ld32(tdP + lane_off + hf * 64 + c2 * 32, dp);
+            tmem_wait_ld();
+#pragma unroll
+            for (int e = 0; e < 32; e += 2) {
+              const float d0 = p[c2 * 32 + e] * (__uint_as_float(dp[e]) - dl[c2 * 32 + e]);
+              const float d1 = p[c2 * 32 + e + 1] * (__uint_as_float(dp[e + 1]) - dl[c2 * 32 + e + 1]);
+              dd[e >> 1] = pack_bf16x2(d0, d1);
+            }
+#pragma unroll
+            for (int ch = 0; ch < 4; ++ch) {
+              const int chunk = (c2 * 4 + ch) ^ (row & 7);
+              *reinterpret_cast<uint4*>(ds_row + (chunk << 4)) =
+                  make_uint4(dd[ch * 4], dd[ch * 4 + 1], dd[ch * 4 + 2], dd[ch * 4 + 3]);
+            }
+          }
+          fence_proxy_async_smem();
+          tc_fence_before();
+          mbar_arrive(bar(kvDsReady));
+        }
+      }
+      // ---- unit epilogue: warps 0-3 write dV, warps 4-7 write dK (scaled) -------------------
+      mbar_wait(bar(kvUnitDone), uc & 1, s_abort);
+      tc_fence_after();
+      {
+        const bool live = (row < kv_len) && (*s_abort == 0);
+        const int tok = kv_start + row;
+        GradT* dst = (hf == 0 ? dv : dk) + ((size_t)tok * Hkv + g) * D;
+        const uint32_t src = (hf == 0 ? tdV : tdK) + lane_off;
+        const float mul = (hf == 0) ? 1.f : scale;
+#pragma unroll
+        for (int c = 0; c < D / 32; ++c) {
+          uint32_t x[32];
+          float y[32];
+          tmem_ld32(src + c * 32, x);
+          tmem_wait_ld();
+#pragma unroll
+          for (int e = 0; e < 32; ++e) y[e] = __uint_as_float(x[e]) * mul;
+          if (live) store_chunk32<GradT>(dst + c * 32, y);
+        }
+      }
+      tc_fence_before();
+      mbar_arrive(bar(kvDkvRead));
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (*s_abort != 0 && tid == 0) set_status(hdr, PK_ERR_TIMEOUT, 3);
+  if (warp == kMmaWarp) tmem_dealloc(tmem, 512);
+}
+
+// =========================================================================================
+// dQ kernel
+// =========================================================================================
+template <int D>
+struct DqSmem {
+  static constexpr int kBoxBytes = 128 * 128;
+  static constexpr int kBoxes = D / 64;
+  static constexpr int kTileBytes = kBoxBytes * kBoxes;
+  static constexpr int kQ = 0;
+  static constexpr int kdO = kTileBytes;
+  static constexpr int kKV0 = 2 * kTileBytes;                // stage s: K then V
+  static constexpr int kStageBytes = 2 * kTileBytes;
+  static constexpr int kBars = kKV0 + 2 * kStageBytes;
+  static constexpr int kMisc = kBars + 16 * 8;
+  static constexpr int kTotal = kMisc + 16;
+};
+
+enum DqBar {
+  dqQFull = 0, dqQEmpty, dqKvFull0, dqKvFull1, dqKvEmpty0, dqKvEmpty1, dqSFull0, dqSFull1,
+  dqDpFull, dqDsReady, dqDone, dqRead, dqNumBars
+};
+
+template <int D, typename GradT>
+__global__ void __launch_bounds__(kWsThreads, 1)
+attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+                   const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_do,
+                   const int4* __restrict__ items, const int32_t* __restrict__ order, int32_t* hdr,
+                   const float* __restrict__ lse, const float* __restrict__ delta,
+                   GradT* __restrict__ dq, int T, int Hq, int Hkv, float scale, float scale_log2) {
+  using L = DqSmem<D>;
+  extern __shared__ __align__(1024) uint8_t smem[];
+  const uint32_t sbase = smem_u32(smem);
+  const uint32_t sQ = sbase + L::kQ, sdO = sbase + L::kdO;
+  const uint32_t bars = sbase + L::kBars;
+  auto bar = [&](int i) { return bars + 8u * (uint32_t)i; };
+  volatile int* s_tmem = reinterpret_cast<volatile int*>(smem + L::kMisc);
+  volatile int* s_abort = s_tmem + 1;
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+
+  if (tid == 0) {
+    mbar_init(bar(dqQFull), 1);
+    mbar_init(bar(dqQEmpty), 1);
+    mbar_init(bar(dqKvFull0), 1);
+    mbar_init(bar(dqKvFull1), 1);
+    mbar_init(bar(dqKvEmpty0), 1);
+    mbar_init(bar(dqKvEmpty1), 1);
+    mbar_init(bar(dqSFull0), 1);
+    mbar_init(bar(dqSFull1), 1);
+    mbar_init(bar(dqDpFull), 1);
+    mbar_init(bar(dqDsReady), kComputeThreads);
+    mbar_init(bar(dqDone), 1);
+    mbar_init(bar(dqRead), kComputeThreads);
+    fence_mbar_init();
+    *s_abort = ((sbase & 1023u) != 0) ? 1 : 0;
+  }
+  if (warp == kMmaWarp) {
+    tmem_alloc(smem_u32(const_cast<int*>(s_tmem)), 512);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = static_cast<uint32_t>(*s_tmem);
+  // [0,128) S buffer 0, [128,256) S buffer 1, [256,384) dP (dS as bf16 reuses its first 64
+  // columns), [384, 384+D) dQ
+  const uint32_t tdP = tmem + 256, tdQ = tmem + 384;
+
+  const int G = Hq / Hkv;
+  const bool plan_ok = (hdr[PK_HDR_PLAN_T] == T);
+  const int n_units = plan_ok ? hdr[PK_HDR_N_ITEMS] * Hq : 0;
+  const int n_cta = gridDim.x, cta = blockIdx.x;
+
+  if (warp == kLoadWarp) {
+    // =============================== loader ===============================================
+    if (lane == 0) {
+      prefetch_tensormap(&tm_q);
+      prefetch_tensormap(&tm_k);
+      prefetch_tensormap(&tm_v);
+      prefetch_tensormap(&tm_do);
+      int gk = 0, uc = 0;
+      for (int r = 0;; ++r, ++uc) {
+        const int u = snake_unit(r, cta, n_cta);
+        if (u >= n_units || *s_abort) break;
+        const int4 it = items[order[u / Hq]];
+        const int h = u % Hq, g = h / G;
+        const int q_start = it.x, kv_start = it.z, kv_len = it.w;
+        const int n_kv = (kv_len + kBN - 1) / kBN;
+        mbar_wait(bar(dqQEmpty), (uc & 1) ^ 1, s_abort);
+        mbar_expect_tx(bar(dqQFull), 2 * L::kTileBytes);
+#pragma unroll
+        for (int b = 0; b < L::kBoxes; ++b) {
+          tma_load_2d(sQ + b * L::kBoxBytes, &tm_q, h * D + b * 64, q_start, bar(dqQFull));
+          tma_load_2d(sdO + b * L::kBoxBytes, &tm_do, h * D + b * 64, q_start, bar(dqQFull));
+        }
+        for (int j = 0; j < n_kv; ++j, ++gk) {
+          const int st = gk & 1;
+          const uint32_t sK = sbase + L::kKV0 + st * L::kStageBytes, sV = sK + L::kTileBytes;
+          mbar_wait(bar(dqKvEmpty0 + st), ((gk >> 1) & 1) ^ 1, s_abort);
+          mbar_expect_tx(bar(dqKvFull0 + st), 2 * L::kTileBytes);
+#pragma unroll
+          for (int b = 0; b < L::kBoxes; ++b) {
+            tma_load_2d(sK + b * L::kBoxBytes, &tm_k, g * D + b * 64, kv_start + j * kBN,
+                        bar(dqKvFull0 + st));
+            tma_load_2d(sV + b * L::kBoxBytes, &tm_v, g * D + b * 64, kv_start + j * kBN,
+                        bar(dqKvFull0 + st));
+          }
+        }
+      }
+    }
+    __syncwarp();
+  } else if (warp == kMmaWarp) {
+    // =============================== MMA issuer ===========================================
+    if (lane == 0) {
+      constexpr uint32_t kIdescS = make_idesc(128, 128, kFmtBF16, kFmtBF16, 0, 0);
+      constexpr uint32_t kIdescDQ = make_idesc(128, D, kFmtBF16, kFmtBF16, 0, 1);
+      int gk = 0, uc = 0;
+      auto issue_s = [&](int g_idx) {       // S = Q K^T into S buffer (g_idx & 1)
+        const uint32_t sK = sbase + L::kKV0 + (g_idx & 1) * L::kStageBytes;
+        const uint32_t tS = tmem + (g_idx & 1) * 128;
+#pragma unroll
+        for (int kk = 0; kk < D / 16; ++kk) {
+          const uint32_t off = (kk / 4) * L::kBoxBytes + (kk % 4) * 32;
+          mma_ss(tS, smem_desc_sw128(sQ + off, 16, 1024), smem_desc_sw128(sK + off, 16, 1024),
+                 kIdescS, kk > 0);
+        }
+        mma_commit(bar(dqSFull0 + (g_idx & 1)));
+      };
+      auto issue_dp = [&](int g_idx) {      // dP = dO V^T
+        const uint32_t sV = sbase + L::kKV0 + (g_idx & 1) * L::kStageBytes + L::kTileBytes;
+#pragma unroll
+        for (int kk = 0; kk < D / 16; ++kk) {
+          const uint32_t off = (kk / 4) * L::kBoxBytes + (kk % 4) * 32;
+          mma_ss(tdP, smem_desc_sw128(sdO + off, 16, 1024), smem_desc_sw128(sV + off, 16, 1024),
+                 kIdescS, kk > 0);
+        }
+        mma_commit(bar(dqDpFull));
+      };
+      for (int r = 0;; ++r, ++uc) {
+        const int u = snake_unit(r, cta, n_cta);
+        if (u >= n_units || *s_abort) break;
+        const int4 it = items[order[u / Hq]];
+        const int n_kv = (it.w + kBN - 1) / kBN;
+        mbar_wait(bar(dqQFull), uc & 1, s_abort);
+        mbar_wait(bar(dqKvFull0 + (gk & 1)), (gk >> 1) & 1, s_abort);
+        tc_fence_after();
+        issue_s(gk);
+        issue_dp(gk);
+        for (int j = 0; j < n_kv; ++j, ++gk) {
+          const int st = gk & 1;
+          const uint32_t sK = sbase + L::kKV0 + st * L::kStageBytes;
+          const bool more = (j + 1 < n_kv);
+          if (more) {   // S(j+1) into the other S buffer: its last reader signalled dS(j-1) already
+            mbar_wait(bar(dqKvFull0 + ((gk + 1) & 1)), ((gk + 1) >> 1) & 1, s_abort);
+            tc_fence_after();
+            issue_s(gk + 1);
+          }
+          mbar_wait(bar(dqDsReady), gk & 1, s_abort);
+          if (j == 0 && uc > 0) mbar_wait(bar(dqRead), (uc - 1) & 1, s_abort);
+          tc_fence_after();
+#pragma unroll
+          for (int kk = 0; kk < kBN / 16; ++kk)   // dQ += dS K   (dS from tensor memory)
+            mma_ts(tdQ, tdP + kk * 8, smem_desc_sw128(sK + kk * 2048, L::kBoxBytes, 1024), kIdescDQ,
+                   (j > 0) | (kk > 0));
+          mma_commit(bar(dqKvEmpty0 + st));
+          if (more) issue_dp(gk + 1);   // overwrites dP/dS(j) after dQ(j) (same pipe, in order)
+        }
+        mma_commit(bar(dqDone));
+        mma_commit(bar(dqQEmpty));
+      }
+    }
+    __syncwarp();
+  } else {
+    // =============================== compute (warps 0-7) ==================================
+    const int row = tid & 127;              // query row inside the tile
+    const int hf = tid >> 7;                // which half of the key columns
+    const uint32_t lane_off = static_cast<uint32_t>((warp & 3) * 32) << 16;
+    int gk = 0, uc = 0;
+    for (int r = 0;; ++r, ++uc) {
+      const int u = snake_unit(r, cta, n_cta);
+      if (u >= n_units || *s_abort) break;
+      const int4 it = items[order[u / Hq]];
+      const int h = u % Hq;
+      const int q_start = it.x, q_len = it.y, kv_len = it.w;
+      const int n_kv = (kv_len + kBN - 1) / kBN;
+      const int tok = q_start + row;
+      const float lse2 = (tok < T) ? lse[(size_t)h * T + tok] * kLog2eWs : 0.f;
+      const float dl = (tok < T) ? delta[(size_t)h * T + tok] : 0.f;
+      for (int j = 0; j < n_kv; ++j, ++gk) {
+        const uint32_t tS = tmem + (gk & 1) * 128;
+        const bool diagonal = (j == n_kv - 1);
+        mbar_wait(bar(dqSFull0 + (gk & 1)), (gk >> 1) & 1, s_abort);
+        tc_fence_after();
+        float p[64];
+        {
+          uint32_t s0[32], s1[32];
+          tmem_ld32(tS + lane_off + hf * 64, s0);
+          tmem_ld32(tS + lane_off + hf * 64 + 32, s1);
+          tmem_wait_ld();
+#pragma unroll
+          for (int c = 0; c < 32; ++c) {
+            const bool ok = !diagonal || (hf * 64 + c <= row);
+            const float x = fast_exp2(fmaf(__uint_as_float(s0[c]), scale_log2, -lse2));
+            p[c] = ok ? x : 0.f;
+          }
+#pragma unroll
+          for (int c = 0; c < 32; ++c) {
+            const bool ok = !diagonal || (hf * 64 + 32 + c <= row);
+            const float x = fast_exp2(fmaf(__uint_as_float(s1[c]), scale_log2, -lse2));
+            p[32 + c] = ok ? x : 0.f;
+          }
+        }
+        mbar_wait(bar(dqDpFull), gk & 1, s_abort);
+        tc_fence_after();
+        uint32_t dd[32];
+#pragma unroll
+        for (int c2 = 0; c2 < 2; ++c2) {
+          uint32_t dp[32];
+          tmem_ld32(tdP + lane_off + hf * 64 + c2 * 32, dp);
+          tmem_wait_ld();
+#pragma unroll
+          for (int e = 0; e < 32; e += 2) {
+            const float d0 = p[c2 * 32 + e] * (__uint_as_float(dp[e]) - dl);
+            const float d1 = p[c2 * 32 + e + 1] * (__uint_as_float(dp[e + 1]) - dl);
+            dd[c2 * 16 + (e >> 1)] = pack_bf16x2(d0, d1);
+          }
+        }
+        // every thread must have read dP before dS overwrites its columns
+        tc_fence_before();
+        compute_bar_sync();
+        tc_fence_after();
+        tmem_st32(tdP + lane_off + hf * 32, dd);
+        tmem_wait_st();
+        tc_fence_before();
+        mbar_arrive(bar(dqDsReady));
+      }
+      // ---- unit epilogue: dQ rows, scaled --------------------------------------------------
+      mbar_wait(bar(dqDone), uc & 1, s_abort);
+      tc_fence_after();
+      {
+        const bool live = (row < q_len) && (*s_abort == 0);
+        GradT* dst = dq + ((size_t)tok * Hq + h) * D + hf * (D / 2);
+#pragma unroll
+        for (int c = 0; c < D / 64; ++c) {
+          uint32_t x[32];
+          float y[32];
+          tmem_ld32(tdQ + lane_off + hf * (D / 2) + c * 32, x);
+          tmem_wait_ld();
+#pragma unroll
+          for (int e = 0; e < 32; ++e) y[e] = __uint_as_float(x[e]) * scale;
+          if (live) store_chunk32<GradT>(dst + c * 32, y);
+        }
+      }
+      tc_fence_before();
+      mbar_arrive(bar(dqRead));
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (*s_abort != 0 && tid == 0) set_status(hdr, PK_ERR_TIMEOUT, 4);
+  if (warp == kMmaWarp) tmem_dealloc(tmem, 512);
+}
+
+template <int D, typename GradT>
+int launch_ws(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
+              const CUtensorMap& tdo, char* ws, const WorkspaceLayout& lay, const float* lse,
+              void* dq, void* dk, void* dv, int T, int Hq, int Hkv, float scale,
+              cudaStream_t stream) {
+  auto kern_kv = attn_bwd_dkv_kernel<D, GradT>;
+  auto kern_q = attn_bwd_dq_kernel<D, GradT>;
+  if (cudaFuncSetAttribute(kern_kv, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           DkvSmem<D>::kTotal) != cudaSuccess ||
+      cudaFuncSetAttribute(kern_q, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           DqSmem<D>::kTotal) != cudaSuccess)
+    return PK_ERR_CUDA;
+  int32_t* hdr = reinterpret_cast<int32_t*>(ws + lay.off[PK_WS_HEADER]);
+  const float* delta = reinterpret_cast<const float*>(ws + lay.off[PK_WS_DELTA]);
+  const int grid = sm_count();
+  {
+    TimedLaunch timed(PK_KERNEL_BWD, stream);
+    kern_kv<<<grid, kWsThreads, DkvSmem<D>::kTotal, stream>>>(
+        tq, tk, tv, tdo, reinterpret_cast<const int4*>(ws + lay.off[PK_WS_BWD_ITEMS]),
+        reinterpret_cast<const int32_t*>(ws + lay.off[PK_WS_BWD_ORDER]), hdr, lse, delta,
+        static_cast<GradT*>(dk), static_cast<GradT*>(dv), T, Hq, Hkv, scale, scale * kLog2eWs);
+  }
+  if (launch_status() != PK_OK) return PK_ERR_CUDA;
+  {
+    TimedLaunch timed(PK_KERNEL_BWD_DQ, stream);
+    kern_q<<<grid, kWsThreads, DqSmem<D>::kTotal, stream>>>(
+        tq, tk, tv, tdo, reinterpret_cast<const int4*>(ws + lay.off[PK_WS_FWD_ITEMS]),
+        reinterpret_cast<const int32_t*>(ws + lay.off[PK_WS_FWD_ORDER]), hdr, lse, delta,
+        static_cast<GradT*>(dq), T, Hq, Hkv, scale, scale * kLog2eWs);
+  }
+  return launch_status();
+}
+
+}  // namespace
+
+int launch_bwd_ws(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
+                  const CUtensorMap& tdo, char* ws, const WorkspaceLayout& lay, const float* lse,
+                  void* dq, void* dk, void* dv, int T, int Hq, int Hkv, int D, int grad_dtype,
+                  float scale, cudaStream_t stream) {
+  if (D == 128) {
+    if (grad_dtype == PK_BF16)
+      return launch_ws<128, __nv_bfloat16>(tq, tk, tv, tdo, ws, lay, lse, dq, dk, dv, T, Hq, Hkv,
+                                           scale, stream);
+    return launch_ws<128, float>(tq, tk, tv, tdo, ws, lay, lse, dq, dk, dv, T, Hq, Hkv, scale,
+                                 stream);
+  }
+  if (grad_dtype == PK_BF16)
+    return launch_ws<64, __nv_bfloat16>(tq, tk, tv, tdo, ws, lay, lse, dq, dk, dv, T, Hq, Hkv,
+                                        scale, stream);
+  return launch_ws<64, float>(tq, tk, tv, tdo, ws, lay, lse, dq, dk, dv, T, Hq, Hkv, scale, stream);
+}
+
+}  // namespace pk

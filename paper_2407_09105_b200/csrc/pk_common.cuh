@@ -2,6 +2,7 @@
 // status word, launch-error helper.  No attention arithmetic lives here.
 #pragma once
 
+#include <cuda.h>
 #include <cuda_runtime.h>
 #include <stddef.h>
 #include <stdint.h>
@@ -97,6 +98,10 @@ struct TimedLaunch {
 int plan_launch(const int32_t* position_ids, int32_t T, int32_t* cu_seqlens, int32_t* n_examples,
                 int32_t* max_seqlen, void* workspace, const WorkspaceLayout& lay,
                 cudaStream_t stream);
+int launch_bwd_ws(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
+                  const CUtensorMap& tdo, char* ws, const WorkspaceLayout& lay, const float* lse,
+                  void* dq, void* dk, void* dv, int T, int Hq, int Hkv, int D, int grad_dtype, float scale,
+                  cudaStream_t stream);
 int rope_table_launch(const int32_t* position_ids, int32_t T, int32_t D, float theta,
                       float* table, cudaStream_t stream);
 
