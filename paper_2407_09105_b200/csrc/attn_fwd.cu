@@ -367,6 +367,9 @@ extern "C" int pk_attn_fwd(const void* q, const void* k, const void* v,
       !make_tile_map_bf16(&tv, v, T, Hkv * D))
     return PK_ERR_CUDA;
 
+  if (!use_rope && (Hq / Hkv) % 2 == 0)   // two query heads of a kv head per CTA, warp-specialised
+    return launch_fwd_ws(tq, tk, tv, ws, lay, out, lse, T, Hq, Hkv, D, out_dtype, softmax_scale,
+                         stream);
 #define PK_FWD(DD, RR, TT) \
   return launch_fwd<DD, RR, TT>(tq, tk, tv, ws, lay, out, lse, T, Hq, Hkv, softmax_scale, stream)
   if (D == 128) {

@@ -1,0 +1,341 @@
+// Warp-specialised forward kernel (no fused RoPE, query heads per kv head even) for sm_100a.
+//
+// One CTA per SM works on TWO query tiles at a time: the same block of <= 128 query rows for two
+// adjacent query heads of one kv head.  Both tiles read the same K and V tiles, so each K/V
+// tile is brought into shared memory once for both, and while the softmax warps of one tile
+// are busy the tensor pipe runs the contractions of the other (ping-pong):
+//   warps 0-3   softmax of tile 0 (one thread per query row, whole row in registers)
+//   warps 4-7   softmax of tile 1
+//   warp  8     issues every tcgen05.mma:  S_t = Q_t K^T  and  O_t += P_t V  (P_t from tensor memory)
+//   warp  9     TMA: the two Q tiles per unit, K/V tiles through a 2-stage ring
+// Tensor memory: [0,128) S_0 / P_0, [128,256) S_1 / P_1, [256,384) O_0, [384,512) O_1.
+// The commit that announces S_t(j) also covers O_t += P_t V of step j-1 (same pipe, in order), so
+// the softmax warps may rescale O_t in tensor memory as soon as they see S_t(j).
+// Units (forward item x head pair) are assigned statically in snake order over the plan's
+// longest-first list.  Every wait is bounded.
+#include <cuda_bf16.h>
+
+#include "attn_common.cuh"
+#include "pk_common.cuh"
+#include "sm100_ptx.cuh"
+#include "tensor_map.cuh"
+
+namespace pk {
+namespace {
+
+using namespace ptx;
+
+constexpr int kFwsThreads = 320;
+constexpr int kFwsMmaWarp = 8;
+constexpr int kFwsLoadWarp = 9;
+constexpr float kLog2eF = 1.4426950408889634f;
+constexpr float kLn2F = 0.6931471805599453f;
+
+__device__ __forceinline__ int snake_unit_f(int r, int cta, int n_cta) {
+  return r * n_cta + ((r & 1) ? (n_cta - 1 - cta) : cta);
+}
+
+template <int D>
+struct FwsSmem {
+  static constexpr int kBoxBytes = 128 * 128;
+  static constexpr int kBoxes = D / 64;
+  static constexpr int kTileBytes = kBoxBytes * kBoxes;
+  static constexpr int kQ0 = 0;                              // Q tile of head pair member 0, then 1
+  static constexpr int kKV0 = 2 * kTileBytes;                // stage s: K then V
+  static constexpr int kStageBytes = 2 * kTileBytes;
+  static constexpr int kBars = kKV0 + 2 * kStageBytes;
+  static constexpr int kMisc = kBars + 16 * 8;
+  static constexpr int kTotal = kMisc + 16;
+};
+
+enum FwsBar {
+  fQFull = 0, fQEmpty, fKvFull0, fKvFull1, fKvEmpty0, fKvEmpty1, fSFull0, fSFull1, fPReady0,
+  fPReady1, fOFull0, fOFull1, fORead0, fORead1, fNumBars
+};
+
+template <typename OutT>
+__device__ __forceinline__ void store_out32(OutT* dst, const uint32_t* r, float scale) {
+  float y[32];
+#pragma unroll
+  for (int e = 0; e < 32; ++e) y[e] = __uint_as_float(r[e]) * scale;
+  store_chunk32<OutT>(dst, y);
+}
+
+template <int D, typename OutT>
+__global__ void __launch_bounds__(kFwsThreads, 1)
+attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+                   const __grid_constant__ CUtensorMap tm_v, const int4* __restrict__ items,
+                   const int32_t* __restrict__ order, int32_t* hdr, OutT* __restrict__ out,
+                   float* __restrict__ lse, int T, int Hq, int Hkv, float scale_log2) {
+  using L = FwsSmem<D>;
+  extern __shared__ __align__(1024) uint8_t smem[];
+  const uint32_t sbase = smem_u32(smem);
+  const uint32_t bars = sbase + L::kBars;
+  auto bar = [&](int i) { return bars + 8u * (uint32_t)i; };
+  volatile int* s_tmem = reinterpret_cast<volatile int*>(smem + L::kMisc);
+  volatile int* s_abort = s_tmem + 1;
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+
+  if (tid == 0) {
+    mbar_init(bar(fQFull), 1);
+    mbar_init(bar(fQEmpty), 1);
+    mbar_init(bar(fKvFull0), 1);
+    mbar_init(bar(fKvFull1), 1);
+    mbar_init(bar(fKvEmpty0), 1);
+    mbar_init(bar(fKvEmpty1), 1);
+    mbar_init(bar(fSFull0), 1);
+    mbar_init(bar(fSFull1), 1);
+    mbar_init(bar(fPReady0), 128);
+    mbar_init(bar(fPReady1), 128);
+    mbar_init(bar(fOFull0), 1);
+    mbar_init(bar(fOFull1), 1);
+    mbar_init(bar(fORead0), 128);
+    mbar_init(bar(fORead1), 128);
+    fence_mbar_init();
+    *s_abort = ((sbase & 1023u) != 0) ? 1 : 0;
+  }
+  if (warp == kFwsMmaWarp) {
+    tmem_alloc(smem_u32(const_cast<int*>(s_tmem)), 512);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = static_cast<uint32_t>(*s_tmem);
+
+  const int G = Hq / Hkv;
+  const int pairs = Hq / 2;
+  const bool plan_ok = (hdr[PK_HDR_PLAN_T] == T);
+  if (!plan_ok && blockIdx.x == 0 && tid == 0) set_status(hdr, PK_ERR_NO_PLAN, T);
+  const int n_units = plan_ok ? hdr[PK_HDR_N_ITEMS] * pairs : 0;
+  const int n_cta = gridDim.x, cta = blockIdx.x;
+
+  if (warp == kFwsLoadWarp) {
+    // =============================== loader ===============================================
+    if (lane == 0) {
+      prefetch_tensormap(&tm_q);
+      prefetch_tensormap(&tm_k);
+      prefetch_tensormap(&tm_v);
+      int gk = 0, uc = 0;
+      for (int r = 0;; ++r, ++uc) {
+        const int u = snake_unit_f(r, cta, n_cta);
+        if (u >= n_units || *s_abort) break;
+        const int4 it = items[order[u / pairs]];
+        const int h0 = (u % pairs) * 2, g = h0 / G;
+        const int q_start = it.x, kv_start = it.z, kv_len = it.w;
+        const int n_kv = (kv_len + kBN - 1) / kBN;
+        mbar_wait(bar(fQEmpty), (uc & 1) ^ 1, s_abort);
+        mbar_expect_tx(bar(fQFull), 2 * L::kTileBytes);
+#pragma unroll
+        for (int t = 0; t < 2; ++t)
+#pragma unroll
+          for (int b = 0; b < L::kBoxes; ++b)
+            tma_load_2d(sbase + L::kQ0 + t * L::kTileBytes + b * L::kBoxBytes, &tm_q,
+                        (h0 + t) * D + b * 64, q_start, bar(fQFull));
+        for (int j = 0; j < n_kv; ++j, ++gk) {
+          const int st = gk & 1;
+          const uint32_t sK = sbase + L::kKV0 + st * L::kStageBytes, sV = sK + L::kTileBytes;
+          mbar_wait(bar(fKvEmpty0 + st), ((gk >> 1) & 1) ^ 1, s_abort);
+          mbar_expect_tx(bar(fKvFull0 + st), 2 * L::kTileBytes);
+#pragma unroll
+          for (int b = 0; b < L::kBoxes; ++b) {
+            tma_load_2d(sK + b * L::kBoxBytes, &tm_k, g * D + b * 64, kv_start + j * kBN,
+                        bar(fKvFull0 + st));
+            tma_load_2d(sV + b * L::kBoxBytes, &tm_v, g * D + b * 64, kv_start + j * kBN,
+                        bar(fKvFull0 + st));
+          }
+        }
+      }
+    }
+    __syncwarp();
+  } else if (warp == kFwsMmaWarp) {
+    // =============================== MMA issuer ===========================================
+    if (lane == 0) {
+      constexpr uint32_t kIdescQK = make_idesc(128, 128, kFmtBF16, kFmtBF16, 0, 0);
+      constexpr uint32_t kIdescPV = make_idesc(128, D, kFmtBF16, kFmtBF16, 0, 1);
+      int gk = 0, uc = 0;
+      auto issue_s = [&](int t, int st) {
+        const uint32_t sQ = sbase + L::kQ0 + t * L::kTileBytes;
+        const uint32_t sK = sbase + L::kKV0 + st * L::kStageBytes;
+#pragma unroll
+        for (int kk = 0; kk < D / 16; ++kk) {
+          const uint32_t off = (kk / 4) * L::kBoxBytes + (kk % 4) * 32;
+          mma_ss(tmem + t * 128, smem_desc_sw128(sQ + off, 16, 1024),
+                 smem_desc_sw128(sK + off, 16, 1024), kIdescQK, kk > 0);
+        }
+        mma_commit(bar(fSFull0 + t));
+      };
+      for (int r = 0;; ++r, ++uc) {
+        const int u = snake_unit_f(r, cta, n_cta);
+        if (u >= n_units || *s_abort) break;
+        const int4 it = items[order[u / pairs]];
+        const int n_kv = (it.w + kBN - 1) / kBN;
+        mbar_wait(bar(fQFull), uc & 1, s_abort);
+        mbar_wait(bar(fKvFull0 + (gk & 1)), (gk >> 1) & 1, s_abort);
+        tc_fence_after();
+        issue_s(0, gk & 1);
+        issue_s(1, gk & 1);
+        for (int j = 0; j < n_kv; ++j, ++gk) {
+          const int st = gk & 1;
+          const uint32_t sV = sbase + L::kKV0 + st * L::kStageBytes + L::kTileBytes;
+          const bool more = (j + 1 < n_kv);
+#pragma unroll
+          for (int t = 0; t < 2; ++t) {
+            mbar_wait(bar(fPReady0 + t), gk & 1, s_abort);
+            if (j == 0 && uc > 0) mbar_wait(bar(fORead0 + t), (uc - 1) & 1, s_abort);
+            tc_fence_after();
+#pragma unroll
+            for (int kk = 0; kk < kBN / 16; ++kk)   // O_t += P_t V
+              mma_ts(tmem + 256 + t * 128, tmem + t * 128 + kk * 8,
+                     smem_desc_sw128(sV + kk * 2048, L::kBoxBytes, 1024), kIdescPV,
+                     (j > 0) | (kk > 0));
+            if (t == 1) mma_commit(bar(fKvEmpty0 + st));
+            if (!more) mma_commit(bar(fOFull0 + t));
+            if (more) {                              // S_t(j+1): P_t(j) was consumed just above
+              if (t == 0) {
+                mbar_wait(bar(fKvFull0 + ((gk + 1) & 1)), ((gk + 1) >> 1) & 1, s_abort);
+                tc_fence_after();
+              }
+              issue_s(t, (gk + 1) & 1);
+            }
+          }
+        }
+        mma_commit(bar(fQEmpty));
+      }
+    }
+    __syncwarp();
+  } else {
+    // =============================== softmax (warps 0-3: tile 0, warps 4-7: tile 1) =======
+    const int t = tid >> 7;
+    const int row = tid & 127;
+    const uint32_t lane_off = static_cast<uint32_t>((warp & 3) * 32) << 16;
+    const uint32_t tS = tmem + t * 128 + lane_off;
+    const uint32_t tO = tmem + 256 + t * 128 + lane_off;
+    int gk = 0, uc = 0;
+    for (int r = 0;; ++r, ++uc) {
+      const int u = snake_unit_f(r, cta, n_cta);
+      if (u >= n_units || *s_abort) break;
+      const int4 it = items[order[u / pairs]];
+      const int h = (u % pairs) * 2 + t;
+      const int q_start = it.x, q_len = it.y, kv_len = it.w;
+      const int n_kv = (kv_len + kBN - 1) / kBN;
+      float m_run = -INFINITY, l_run = 0.f;
+      for (int j = 0; j < n_kv; ++j, ++gk) {
+        mbar_wait(bar(fSFull0 + t), gk & 1, s_abort);
+        tc_fence_after();
+        uint32_t s[128];
+#pragma unroll
+        for (int c = 0; c < 4; ++c) tmem_ld32(tS + c * 32, s + c * 32);
+        tmem_wait_ld();
+        if (j == n_kv - 1) {   // diagonal tile: keys after the query row are masked
+#pragma unroll
+          for (int c = 0; c < 128; ++c)
+            if (c > row) s[c] = 0xff800000u;   // -inf
+        }
+        float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};   // independent chains
+#pragma unroll
+        for (int c = 0; c < 128; c += 4) {
+#pragma unroll
+          for (int e = 0; e < 4; ++e) mx4[e] = fmaxf(mx4[e], __uint_as_float(s[c + e]));
+        }
+        const float row_m = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * scale_log2;
+        // the reference maximum only moves when the row maximum exceeds it by more than 2^8, so
+        // that the running O rarely needs rescaling; P then stays below 2^8
+        const bool changed = row_m > m_run + 8.f;          // true on the first tile (m_run = -inf)
+        const float m_new = changed ? row_m : m_run;
+        const float alpha = changed ? fast_exp2(m_run - m_new) : 1.f;   // 0 on the first tile
+        float sum4[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {   // P leaves in two 64-column pieces to bound registers
+          uint32_t p[32];
+#pragma unroll
+          for (int c = 0; c < 64; c += 4) {
+            const float p0 = fast_exp2(fmaf(__uint_as_float(s[half * 64 + c]), scale_log2, -m_new));
+            const float p1 = fast_exp2(fmaf(__uint_as_float(s[half * 64 + c + 1]), scale_log2, -m_new));
+            const float p2 = fast_exp2(fmaf(__uint_as_float(s[half * 64 + c + 2]), scale_log2, -m_new));
+            const float p3 = fast_exp2(fmaf(__uint_as_float(s[half * 64 + c + 3]), scale_log2, -m_new));
+            sum4[0] += p0; sum4[1] += p1; sum4[2] += p2; sum4[3] += p3;
+            p[c >> 1] = pack_bf16x2(p0, p1);
+            p[(c >> 1) + 1] = pack_bf16x2(p2, p3);
+          }
+          tmem_st32(tS + half * 32, p);
+        }
+        l_run = l_run * alpha + ((sum4[0] + sum4[1]) + (sum4[2] + sum4[3]));
+        m_run = m_new;
+        // O_t of step j-1 is complete (its contraction precedes S_t(j) on the tensor pipe)
+        if (j > 0 && __any_sync(0xffffffffu, changed)) {
+#pragma unroll
+          for (int c = 0; c < D / 32; ++c) {
+            uint32_t o[32];
+            tmem_ld32(tO + c * 32, o);
+            tmem_wait_ld();
+#pragma unroll
+            for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
+            tmem_st32(tO + c * 32, o);
+          }
+        }
+        tmem_wait_st();
+        tc_fence_before();
+        mbar_arrive(bar(fPReady0 + t));
+      }
+      // ---- epilogue: O / l and lse ---------------------------------------------------------
+      mbar_wait(bar(fOFull0 + t), uc & 1, s_abort);
+      tc_fence_after();
+      {
+        const bool live = (row < q_len) && (*s_abort == 0);
+        const float inv_l = 1.f / l_run;
+        if (live) lse[(size_t)h * T + q_start + row] = (m_run + log2f(l_run)) * kLn2F;
+        OutT* orow = out + ((size_t)(q_start + row) * Hq + h) * D;
+#pragma unroll
+        for (int c = 0; c < D / 32; ++c) {
+          uint32_t o[32];
+          tmem_ld32(tO + c * 32, o);
+          tmem_wait_ld();
+          if (live) store_out32<OutT>(orow + c * 32, o, inv_l);
+        }
+      }
+      tc_fence_before();
+      mbar_arrive(bar(fORead0 + t));
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (*s_abort != 0 && tid == 0) set_status(hdr, PK_ERR_TIMEOUT, 5);
+  if (warp == kFwsMmaWarp) tmem_dealloc(tmem, 512);
+}
+
+template <int D, typename OutT>
+int launch_fws(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, char* ws,
+               const WorkspaceLayout& lay, void* out, float* lse, int T, int Hq, int Hkv,
+               float scale, cudaStream_t stream) {
+  auto kern = attn_fwd_ws_kernel<D, OutT>;
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           FwsSmem<D>::kTotal) != cudaSuccess)
+    return PK_ERR_CUDA;
+  int32_t* hdr = reinterpret_cast<int32_t*>(ws + lay.off[PK_WS_HEADER]);
+  TimedLaunch timed(PK_KERNEL_FWD, stream);
+  kern<<<sm_count(), kFwsThreads, FwsSmem<D>::kTotal, stream>>>(
+      tq, tk, tv, reinterpret_cast<const int4*>(ws + lay.off[PK_WS_FWD_ITEMS]),
+      reinterpret_cast<const int32_t*>(ws + lay.off[PK_WS_FWD_ORDER]), hdr,
+      static_cast<OutT*>(out), lse, T, Hq, Hkv, scale * kLog2eF);
+  return launch_status();
+}
+
+}  // namespace
+
+int launch_fwd_ws(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, char* ws,
+                  const WorkspaceLayout& lay, void* out, float* lse, int T, int Hq, int Hkv, int D,
+                  int out_dtype, float scale, cudaStream_t stream) {
+  if (D == 128) {
+    if (out_dtype == PK_BF16)
+      return launch_fws<128, __nv_bfloat16>(tq, tk, tv, ws, lay, out, lse, T, Hq, Hkv, scale, stream);
+    return launch_fws<128, float>(tq, tk, tv, ws, lay, out, lse, T, Hq, Hkv, scale, stream);
+  }
+  if (out_dtype == PK_BF16)
+    return launch_fws<64, __nv_bfloat16>(tq, tk, tv, ws, lay, out, lse, T, Hq, Hkv, scale, stream);
+  return launch_fws<64, float>(tq, tk, tv, ws, lay, out, lse, T, Hq, Hkv, scale, stream);
+}
+
+}  // namespace pk

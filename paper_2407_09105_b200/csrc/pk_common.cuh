@@ -102,6 +102,9 @@ int launch_bwd_ws(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMa
                   const CUtensorMap& tdo, char* ws, const WorkspaceLayout& lay, const float* lse,
                   void* dq, void* dk, void* dv, int T, int Hq, int Hkv, int D, int grad_dtype, float scale,
                   cudaStream_t stream);
+int launch_fwd_ws(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, char* ws,
+                  const WorkspaceLayout& lay, void* out, float* lse, int T, int Hq, int Hkv, int D,
+                  int out_dtype, float scale, cudaStream_t stream);
 int rope_table_launch(const int32_t* position_ids, int32_t T, int32_t D, float theta,
                       float* table, cudaStream_t stream);
 
