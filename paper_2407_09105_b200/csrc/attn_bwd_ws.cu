@@ -15,8 +15,10 @@
 // Both recompute S and dP (7 contractions per tile pair instead of 5), both are bitwise
 // reproducible, and both never visit a tile outside an example's causal block.
 //
-// Roles (320 threads): warps 0-7 compute (lane = tensor-memory row; warps 0-3 take columns
-// 0..63, warps 4-7 columns 64..127), warp 8 issues every tcgen05.mma, warp 9 drives TMA.
+// Roles: 16 compute warps (lane = tensor-memory row; warp w works on columns
+// [32*(w/4), 32*(w/4)+32) of the rows of lane quarter w%4 -- many warps, because the compute
+// phases are bound by latency, not by issue or special-function throughput), one warp that
+// issues every tcgen05.mma, one warp that drives TMA.
 // Units are assigned statically: CTA c takes positions c, 2P-1-c, 2P+c, ... of the plan's
 // longest-first order, so the roles enumerate the same sequence without talking to each other.
 // Every wait is bounded; on expiry an abort flag makes all later waits return at once.
@@ -32,10 +34,15 @@ namespace {
 
 using namespace ptx;
 
-constexpr int kWsThreads = 320;
-constexpr int kComputeThreads = 256;
-constexpr int kMmaWarp = 8;
-constexpr int kLoadWarp = 9;
+#ifndef PK_BWD_COMPUTE_THREADS
+#define PK_BWD_COMPUTE_THREADS 512
+#endif
+constexpr int kComputeThreads = PK_BWD_COMPUTE_THREADS;   // 256 or 512
+constexpr int kNQ = kComputeThreads / 128;                // column groups per tile row
+constexpr int kCW = 128 / kNQ;                            // columns per compute thread
+constexpr int kWsThreads = kComputeThreads + 64;
+constexpr int kMmaWarp = kComputeThreads / 32;
+constexpr int kLoadWarp = kMmaWarp + 1;
 constexpr float kLog2eWs = 1.4426950408889634f;
 
 // position in the longest-first order of the r-th unit of this CTA (snake over the rounds)
@@ -43,7 +50,7 @@ __device__ __forceinline__ int snake_unit(int r, int cta, int n_cta) {
   return r * n_cta + ((r & 1) ? (n_cta - 1 - cta) : cta);
 }
 __device__ __forceinline__ void compute_bar_sync() {
-  asm volatile("bar.sync 1, 256;" ::: "memory");
+  asm volatile("bar.sync 1, %0;" ::"n"(kComputeThreads) : "memory");
 }
 
 // =========================================================================================
@@ -259,9 +266,9 @@ attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     }
     __syncwarp();
   } else {
-    // =============================== compute (warps 0-7) ==================================
+    // =============================== compute ===============================================
     const int row = tid & 127;              // key row inside the block
-    const int hf = tid >> 7;                // which half of the query columns
+    const int qd = tid >> 7;                // which group of kCW query columns
     const uint32_t lane_off = static_cast<uint32_t>((warp & 3) * 32) << 16;
     int gs = 0, uc = 0;
     for (int r = 0;; ++r, ++uc) {
@@ -276,41 +283,45 @@ attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           const int st = gs & 1;
           const int q_left = q_len - i * kBM;
           const int col_min = (i == 0) ? row : 0;
-          const float* lse2 = s_lse + st * 128 + hf * 64;
-          const float* dl = s_delta + st * 128 + hf * 64;
+          const float4* lse4 = reinterpret_cast<const float4*>(s_lse + st * 128 + qd * kCW);
+          const float4* dl4 = reinterpret_cast<const float4*>(s_delta + st * 128 + qd * kCW);
           mbar_wait(bar(kvQFull0 + st), (gs >> 1) & 1, s_abort);   // lse / delta rows visible
           mbar_wait(bar(kvSFull), gs & 1, s_abort);
           tc_fence_after();
-          float p[64];
+          float p[kCW];
           {
-            uint32_t s0[32], s1[32];
-            tmem_ld32(tS + lane_off + hf * 64, s0);
-            tmem_ld32(tS + lane_off + hf * 64 + 32, s1);
+            uint32_t sv[kCW];
+#pragma unroll
+            for (int c0 = 0; c0 < kCW; c0 += 32) tmem_ld32(tS + lane_off + qd * kCW + c0, sv + c0);
             tmem_wait_ld();
 #pragma unroll
-            for (int c = 0; c < 32; ++c) {
-              const int col = hf * 64 + c;
-              const bool ok = (col >= col_min) && (col < q_left);
-              const float x = fast_exp2(fmaf(__uint_as_float(s0[c]), scale_log2, -lse2[c]));
-              p[c] = ok ? x : 0.f;
+            for (int c = 0; c < kCW; c += 4) {
+              const float4 l4 = lse4[c >> 2];
+              p[c] = fast_exp2(fmaf(__uint_as_float(sv[c]), scale_log2, -l4.x));
+              p[c + 1] = fast_exp2(fmaf(__uint_as_float(sv[c + 1]), scale_log2, -l4.y));
+              p[c + 2] = fast_exp2(fmaf(__uint_as_float(sv[c + 2]), scale_log2, -l4.z));
+              p[c + 3] = fast_exp2(fmaf(__uint_as_float(sv[c + 3]), scale_log2, -l4.w));
             }
+            // masks are needed only on the diagonal tile (causal) and on a last, partial tile
+            // (query rows past the example end); interior tiles skip the compares
+            if (i == 0 || q_left < kBM) {
 #pragma unroll
-            for (int c = 0; c < 32; ++c) {
-              const int col = hf * 64 + 32 + c;
-              const bool ok = (col >= col_min) && (col < q_left);
-              const float x = fast_exp2(fmaf(__uint_as_float(s1[c]), scale_log2, -lse2[32 + c]));
-              p[32 + c] = ok ? x : 0.f;
+              for (int c = 0; c < kCW; ++c) {
+                const int col = qd * kCW + c;
+                if (!((col >= col_min) && (col < q_left))) p[c] = 0.f;
+              }
             }
           }
-          // both halves must have read S before P overwrites its columns
+          // every column group must have read S before P overwrites its columns
           tc_fence_before();
           compute_bar_sync();
           tc_fence_after();
           {
-            uint32_t pp[32];
+            uint32_t pp[kCW / 2];
 #pragma unroll
-            for (int c = 0; c < 32; ++c) pp[c] = pack_bf16x2(p[2 * c], p[2 * c + 1]);
-            tmem_st32(tS + lane_off + hf * 32, pp);
+            for (int c = 0; c < kCW / 2; ++c) pp[c] = pack_bf16x2(p[2 * c], p[2 * c + 1]);
+            if (kCW == 64) tmem_st32(tS + lane_off + qd * (kCW / 2), pp);
+            else tmem_st16(tS + lane_off + qd * (kCW / 2), pp);
             tmem_wait_st();
           }
           tc_fence_before();
@@ -318,21 +329,29 @@ attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 
           mbar_wait(bar(kvDpFull), gs & 1, s_abort);
           tc_fence_after();
-          uint8_t* ds_row = smem + L::kdS + hf * L::kBoxBytes + row * 128;
+          // dS^T row `row`, query columns [qd*kCW, +kCW): box (qd*kCW)/64, 16-byte chunks from
+          // ((qd*kCW)%64)/8 on
+          uint8_t* ds_row = smem + L::kdS + ((qd * kCW) / 64) * L::kBoxBytes + row * 128;
+          constexpr int kChunk0 = 0;
 #pragma unroll
-          for (int c2 = 0; c2 < 2; ++c2) {
+          for (int c2 = 0; c2 < kCW / 32; ++c2) {
             uint32_t dp[32], dd[16];
-            tmem_ld32(tdP + lane_off + hf * 64 + c2 * 32, dp);
+            tmem_ld32(tdP + lane_off + qd * kCW + c2 * 32, dp);
             tmem_wait_ld();
 #pragma unroll
-            for (int e = 0; e < 32; e += 2) {
-              const float d0 = p[c2 * 32 + e] * (__uint_as_float(dp[e]) - dl[c2 * 32 + e]);
-              const float d1 = p[c2 * 32 + e + 1] * (__uint_as_float(dp[e + 1]) - dl[c2 * 32 + e + 1]);
+            for (int e = 0; e < 32; e += 4) {
+              const float4 d4 = dl4[(c2 * 32 + e) >> 2];
+              const float d0 = p[c2 * 32 + e] * (__uint_as_float(dp[e]) - d4.x);
+              const float d1 = p[c2 * 32 + e + 1] * (__uint_as_float(dp[e + 1]) - d4.y);
+              const float d2 = p[c2 * 32 + e + 2] * (__uint_as_float(dp[e + 2]) - d4.z);
+              const float d3 = p[c2 * 32 + e + 3] * (__uint_as_float(dp[e + 3]) - d4.w);
               dd[e >> 1] = pack_bf16x2(d0, d1);
+              dd[(e >> 1) + 1] = pack_bf16x2(d2, d3);
             }
+            const int chunk_base = kChunk0 + ((qd * kCW) % 64) / 8 + c2 * 4;
 #pragma unroll
             for (int ch = 0; ch < 4; ++ch) {
-              const int chunk = (c2 * 4 + ch) ^ (row & 7);
+              const int chunk = (chunk_base + ch) ^ (row & 7);
               *reinterpret_cast<uint4*>(ds_row + (chunk << 4)) =
                   make_uint4(dd[ch * 4], dd[ch * 4 + 1], dd[ch * 4 + 2], dd[ch * 4 + 3]);
             }
@@ -342,17 +361,21 @@ attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           mbar_arrive(bar(kvDsReady));
         }
       }
-      // ---- unit epilogue: warps 0-3 write dV, warps 4-7 write dK (scaled) -------------------
+      // ---- unit epilogue: the first half of the column groups writes dV, the second dK ------
       mbar_wait(bar(kvUnitDone), uc & 1, s_abort);
       tc_fence_after();
       {
+        constexpr int kHalfGroups = kNQ / 2;               // groups per output tensor
+        constexpr int kEpiCols = D / kHalfGroups;          // columns each thread writes
+        const bool is_dv = qd < kHalfGroups;
+        const int col0 = (qd % kHalfGroups) * kEpiCols;
         const bool live = (row < kv_len) && (*s_abort == 0);
         const int tok = kv_start + row;
-        GradT* dst = (hf == 0 ? dv : dk) + ((size_t)tok * Hkv + g) * D;
-        const uint32_t src = (hf == 0 ? tdV : tdK) + lane_off;
-        const float mul = (hf == 0) ? 1.f : scale;
+        GradT* dst = (is_dv ? dv : dk) + ((size_t)tok * Hkv + g) * D + col0;
+        const uint32_t src = (is_dv ? tdV : tdK) + lane_off + col0;
+        const float mul = is_dv ? 1.f : scale;
 #pragma unroll
-        for (int c = 0; c < D / 32; ++c) {
+        for (int c = 0; c < kEpiCols / 32; ++c) {
           uint32_t x[32];
           float y[32];
           tmem_ld32(src + c * 32, x);
@@ -383,16 +406,21 @@ struct DqSmem {
   static constexpr int kTileBytes = kBoxBytes * kBoxes;
   static constexpr int kQ = 0;
   static constexpr int kdO = kTileBytes;
-  static constexpr int kKV0 = 2 * kTileBytes;                // stage s: K then V
-  static constexpr int kStageBytes = 2 * kTileBytes;
-  static constexpr int kBars = kKV0 + 2 * kStageBytes;
-  static constexpr int kMisc = kBars + 16 * 8;
+  // K tiles live from S(j) to dQ(j), V tiles only for dP(j): separate rings, K one stage
+  // deeper, so that the loads run two steps ahead of the contractions
+  static constexpr int kKStages = 3;
+  static constexpr int kVStages = 2;
+  static constexpr int kK0 = 2 * kTileBytes;
+  static constexpr int kV0 = kK0 + kKStages * kTileBytes;
+  static constexpr int kBars = kV0 + kVStages * kTileBytes;
+  static constexpr int kMisc = kBars + 24 * 8;
   static constexpr int kTotal = kMisc + 16;
 };
 
 enum DqBar {
-  dqQFull = 0, dqQEmpty, dqKvFull0, dqKvFull1, dqKvEmpty0, dqKvEmpty1, dqSFull0, dqSFull1,
-  dqDpFull, dqDsReady, dqDone, dqRead, dqNumBars
+  dqQFull = 0, dqQEmpty, dqKFull0, dqKFull1, dqKFull2, dqKEmpty0, dqKEmpty1, dqKEmpty2, dqVFull0,
+  dqVFull1, dqVEmpty0, dqVEmpty1, dqSFull0, dqSFull1, dqDpFull, dqDsReady, dqDone, dqRead,
+  dqNumBars
 };
 
 template <int D, typename GradT>
@@ -416,10 +444,7 @@ attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
   if (tid == 0) {
     mbar_init(bar(dqQFull), 1);
     mbar_init(bar(dqQEmpty), 1);
-    mbar_init(bar(dqKvFull0), 1);
-    mbar_init(bar(dqKvFull1), 1);
-    mbar_init(bar(dqKvEmpty0), 1);
-    mbar_init(bar(dqKvEmpty1), 1);
+    for (int i = dqKFull0; i <= dqVEmpty1; ++i) mbar_init(bar(i), 1);
     mbar_init(bar(dqSFull0), 1);
     mbar_init(bar(dqSFull1), 1);
     mbar_init(bar(dqDpFull), 1);
@@ -469,17 +494,21 @@ attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
           tma_load_2d(sdO + b * L::kBoxBytes, &tm_do, h * D + b * 64, q_start, bar(dqQFull));
         }
         for (int j = 0; j < n_kv; ++j, ++gk) {
-          const int st = gk & 1;
-          const uint32_t sK = sbase + L::kKV0 + st * L::kStageBytes, sV = sK + L::kTileBytes;
-          mbar_wait(bar(dqKvEmpty0 + st), ((gk >> 1) & 1) ^ 1, s_abort);
-          mbar_expect_tx(bar(dqKvFull0 + st), 2 * L::kTileBytes);
+          const int ks = gk % L::kKStages, vs = gk % L::kVStages;
+          const uint32_t sK = sbase + L::kK0 + ks * L::kTileBytes;
+          const uint32_t sV = sbase + L::kV0 + vs * L::kTileBytes;
+          mbar_wait(bar(dqKEmpty0 + ks), ((gk / L::kKStages) & 1) ^ 1, s_abort);
+          mbar_expect_tx(bar(dqKFull0 + ks), L::kTileBytes);
 #pragma unroll
-          for (int b = 0; b < L::kBoxes; ++b) {
+          for (int b = 0; b < L::kBoxes; ++b)
             tma_load_2d(sK + b * L::kBoxBytes, &tm_k, g * D + b * 64, kv_start + j * kBN,
-                        bar(dqKvFull0 + st));
+                        bar(dqKFull0 + ks));
+          mbar_wait(bar(dqVEmpty0 + vs), ((gk / L::kVStages) & 1) ^ 1, s_abort);
+          mbar_expect_tx(bar(dqVFull0 + vs), L::kTileBytes);
+#pragma unroll
+          for (int b = 0; b < L::kBoxes; ++b)
             tma_load_2d(sV + b * L::kBoxBytes, &tm_v, g * D + b * 64, kv_start + j * kBN,
-                        bar(dqKvFull0 + st));
-          }
+                        bar(dqVFull0 + vs));
         }
       }
     }
@@ -491,8 +520,11 @@ attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
       constexpr uint32_t kIdescDQ = make_idesc(128, D, kFmtBF16, kFmtBF16, 0, 1);
       int gk = 0, uc = 0;
       auto issue_s = [&](int g_idx) {       // S = Q K^T into S buffer (g_idx & 1)
-        const uint32_t sK = sbase + L::kKV0 + (g_idx & 1) * L::kStageBytes;
+        const int ks = g_idx % L::kKStages;
+        const uint32_t sK = sbase + L::kK0 + ks * L::kTileBytes;
         const uint32_t tS = tmem + (g_idx & 1) * 128;
+        mbar_wait(bar(dqKFull0 + ks), (g_idx / L::kKStages) & 1, s_abort);
+        tc_fence_after();
 #pragma unroll
         for (int kk = 0; kk < D / 16; ++kk) {
           const uint32_t off = (kk / 4) * L::kBoxBytes + (kk % 4) * 32;
@@ -501,8 +533,11 @@ attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         }
         mma_commit(bar(dqSFull0 + (g_idx & 1)));
       };
-      auto issue_dp = [&](int g_idx) {      // dP = dO V^T
-        const uint32_t sV = sbase + L::kKV0 + (g_idx & 1) * L::kStageBytes + L::kTileBytes;
+      auto issue_dp = [&](int g_idx) {      // dP = dO V^T; the V stage is free once it completes
+        const int vs = g_idx % L::kVStages;
+        const uint32_t sV = sbase + L::kV0 + vs * L::kTileBytes;
+        mbar_wait(bar(dqVFull0 + vs), (g_idx / L::kVStages) & 1, s_abort);
+        tc_fence_after();
 #pragma unroll
         for (int kk = 0; kk < D / 16; ++kk) {
           const uint32_t off = (kk / 4) * L::kBoxBytes + (kk % 4) * 32;
@@ -510,6 +545,7 @@ attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                  kIdescS, kk > 0);
         }
         mma_commit(bar(dqDpFull));
+        mma_commit(bar(dqVEmpty0 + vs));
       };
       for (int r = 0;; ++r, ++uc) {
         const int u = snake_unit(r, cta, n_cta);
@@ -517,19 +553,14 @@ attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         const int4 it = items[order[u / Hq]];
         const int n_kv = (it.w + kBN - 1) / kBN;
         mbar_wait(bar(dqQFull), uc & 1, s_abort);
-        mbar_wait(bar(dqKvFull0 + (gk & 1)), (gk >> 1) & 1, s_abort);
         tc_fence_after();
         issue_s(gk);
         issue_dp(gk);
         for (int j = 0; j < n_kv; ++j, ++gk) {
-          const int st = gk & 1;
-          const uint32_t sK = sbase + L::kKV0 + st * L::kStageBytes;
+          const int ks = gk % L::kKStages;
+          const uint32_t sK = sbase + L::kK0 + ks * L::kTileBytes;
           const bool more = (j + 1 < n_kv);
-          if (more) {   // S(j+1) into the other S buffer: its last reader signalled dS(j-1) already
-            mbar_wait(bar(dqKvFull0 + ((gk + 1) & 1)), ((gk + 1) >> 1) & 1, s_abort);
-            tc_fence_after();
-            issue_s(gk + 1);
-          }
+          if (more) issue_s(gk + 1);   // other S buffer: its last reader signalled dS(j-1) already
           mbar_wait(bar(dqDsReady), gk & 1, s_abort);
           if (j == 0 && uc > 0) mbar_wait(bar(dqRead), (uc - 1) & 1, s_abort);
           tc_fence_after();
@@ -537,7 +568,7 @@ attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
           for (int kk = 0; kk < kBN / 16; ++kk)   // dQ += dS K   (dS from tensor memory)
             mma_ts(tdQ, tdP + kk * 8, smem_desc_sw128(sK + kk * 2048, L::kBoxBytes, 1024), kIdescDQ,
                    (j > 0) | (kk > 0));
-          mma_commit(bar(dqKvEmpty0 + st));
+          mma_commit(bar(dqKEmpty0 + ks));
           if (more) issue_dp(gk + 1);   // overwrites dP/dS(j) after dQ(j) (same pipe, in order)
         }
         mma_commit(bar(dqDone));
@@ -546,9 +577,9 @@ attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
     }
     __syncwarp();
   } else {
-    // =============================== compute (warps 0-7) ==================================
+    // =============================== compute ===============================================
     const int row = tid & 127;              // query row inside the tile
-    const int hf = tid >> 7;                // which half of the key columns
+    const int qd = tid >> 7;                // which group of kCW key columns
     const uint32_t lane_off = static_cast<uint32_t>((warp & 3) * 32) << 16;
     int gk = 0, uc = 0;
     for (int r = 0;; ++r, ++uc) {
@@ -563,35 +594,30 @@ attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
       const float dl = (tok < T) ? delta[(size_t)h * T + tok] : 0.f;
       for (int j = 0; j < n_kv; ++j, ++gk) {
         const uint32_t tS = tmem + (gk & 1) * 128;
-        const bool diagonal = (j == n_kv - 1);
         mbar_wait(bar(dqSFull0 + (gk & 1)), (gk >> 1) & 1, s_abort);
         tc_fence_after();
-        float p[64];
+        float p[kCW];
         {
-          uint32_t s0[32], s1[32];
-          tmem_ld32(tS + lane_off + hf * 64, s0);
-          tmem_ld32(tS + lane_off + hf * 64 + 32, s1);
+          uint32_t sv[kCW];
+#pragma unroll
+          for (int c0 = 0; c0 < kCW; c0 += 32) tmem_ld32(tS + lane_off + qd * kCW + c0, sv + c0);
           tmem_wait_ld();
 #pragma unroll
-          for (int c = 0; c < 32; ++c) {
-            const bool ok = !diagonal || (hf * 64 + c <= row);
-            const float x = fast_exp2(fmaf(__uint_as_float(s0[c]), scale_log2, -lse2));
-            p[c] = ok ? x : 0.f;
-          }
+          for (int c = 0; c < kCW; ++c)
+            p[c] = fast_exp2(fmaf(__uint_as_float(sv[c]), scale_log2, -lse2));
+          if (j == n_kv - 1) {   // only the diagonal tile needs the causal mask
 #pragma unroll
-          for (int c = 0; c < 32; ++c) {
-            const bool ok = !diagonal || (hf * 64 + 32 + c <= row);
-            const float x = fast_exp2(fmaf(__uint_as_float(s1[c]), scale_log2, -lse2));
-            p[32 + c] = ok ? x : 0.f;
+            for (int c = 0; c < kCW; ++c)
+              if (qd * kCW + c > row) p[c] = 0.f;
           }
         }
         mbar_wait(bar(dqDpFull), gk & 1, s_abort);
         tc_fence_after();
-        uint32_t dd[32];
+        uint32_t dd[kCW / 2];
 #pragma unroll
-        for (int c2 = 0; c2 < 2; ++c2) {
+        for (int c2 = 0; c2 < kCW / 32; ++c2) {
           uint32_t dp[32];
-          tmem_ld32(tdP + lane_off + hf * 64 + c2 * 32, dp);
+          tmem_ld32(tdP + lane_off + qd * kCW + c2 * 32, dp);
           tmem_wait_ld();
 #pragma unroll
           for (int e = 0; e < 32; e += 2) {
@@ -604,22 +630,23 @@ attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         tc_fence_before();
         compute_bar_sync();
         tc_fence_after();
-        tmem_st32(tdP + lane_off + hf * 32, dd);
+        if (kCW == 64) tmem_st32(tdP + lane_off + qd * (kCW / 2), dd);
+        else tmem_st16(tdP + lane_off + qd * (kCW / 2), dd);
         tmem_wait_st();
         tc_fence_before();
         mbar_arrive(bar(dqDsReady));
       }
-      // ---- unit epilogue: dQ rows, scaled --------------------------------------------------
+      // ---- unit epilogue: dQ rows, scaled (column groups 0 and 1 write half a row each) -----
       mbar_wait(bar(dqDone), uc & 1, s_abort);
       tc_fence_after();
-      {
+      if (qd < 2) {
         const bool live = (row < q_len) && (*s_abort == 0);
-        GradT* dst = dq + ((size_t)tok * Hq + h) * D + hf * (D / 2);
+        GradT* dst = dq + ((size_t)tok * Hq + h) * D + qd * (D / 2);
 #pragma unroll
         for (int c = 0; c < D / 64; ++c) {
           uint32_t x[32];
           float y[32];
-          tmem_ld32(tdQ + lane_off + hf * (D / 2) + c * 32, x);
+          tmem_ld32(tdQ + lane_off + qd * (D / 2) + c * 32, x);
           tmem_wait_ld();
 #pragma unroll
           for (int e = 0; e < 32; ++e) y[e] = __uint_as_float(x[e]) * scale;
