@@ -313,7 +313,7 @@ def main():
     executed = ((8 if split else 10) * D * Hq * w.causal_pairs) / (bwd_ms * 1e-3) / 1e12
     fwd_tflops = w.useful_flops_fwd / (fwd_ms * 1e-3) / 1e12
     roofline = {
-        "kernel": "attn_bwd_kernel", "bound": "tensor", "achieved": bwd_tflops,
+        "kernel": "attn_bwd_dkv_kernel" if split else "attn_bwd_kernel", "bound": "tensor", "achieved": bwd_tflops,
         "peak": peaks["sustained"], "peak_kind": f"bf16 sustained, {peaks['source']}",
         "peak_burst": peaks["burst"], "unit": "TFLOP/s", "frac": bwd_tflops / peaks["sustained"],
         "traffic": (None if NCU_BWD_DRAM_BYTES_PER_PAIR is None
