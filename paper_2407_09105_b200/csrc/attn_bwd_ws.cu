@@ -188,29 +188,37 @@ attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     }
   } else if (warp == kMmaWarp) {
     // =============================== MMA issuer ===========================================
-    if (lane == 0) {
+    // The whole warp walks the schedule (so that addresses and descriptors stay warp-uniform);
+    // one elected lane issues the tensor-core instructions.
+    {
       constexpr uint32_t kIdescS = make_idesc(128, 128, kFmtBF16, kFmtBF16, 0, 0);
       constexpr uint32_t kIdescKV = make_idesc(128, D, kFmtBF16, kFmtBF16, 0, 1);
+      const bool leader = elect_one();
+      const uint32_t k_lo = desc_lo(sK, 16), v_lo = desc_lo(sV, 16), ds_lo = desc_lo(sdS, 16);
       int gs = 0, uc = 0;
       auto issue_s = [&](int st) {
-        const uint32_t sQ = sbase + L::kQ0 + st * L::kStageBytes;
+        const uint32_t q_lo = desc_lo(sbase + L::kQ0 + st * L::kStageBytes, 16);
+        if (leader) {
 #pragma unroll
-        for (int kk = 0; kk < D / 16; ++kk) {
-          const uint32_t off = (kk / 4) * L::kBoxBytes + (kk % 4) * 32;
-          mma_ss(tS, smem_desc_sw128(sK + off, 16, 1024), smem_desc_sw128(sQ + off, 16, 1024),
-                 kIdescS, kk > 0);
+          for (int kk = 0; kk < D / 16; ++kk) {
+            const uint32_t off = ((kk / 4) * L::kBoxBytes + (kk % 4) * 32) >> 4;
+            mma_ss(tS, desc_from_lo(k_lo + off), desc_from_lo(q_lo + off), kIdescS, kk > 0);
+          }
+          mma_commit(bar(kvSFull));
         }
-        mma_commit(bar(kvSFull));
+        __syncwarp();
       };
       auto issue_dp = [&](int st) {
-        const uint32_t sdO = sbase + L::kQ0 + st * L::kStageBytes + L::kTileBytes;
+        const uint32_t do_lo = desc_lo(sbase + L::kQ0 + st * L::kStageBytes + L::kTileBytes, 16);
+        if (leader) {
 #pragma unroll
-        for (int kk = 0; kk < D / 16; ++kk) {
-          const uint32_t off = (kk / 4) * L::kBoxBytes + (kk % 4) * 32;
-          mma_ss(tdP, smem_desc_sw128(sV + off, 16, 1024), smem_desc_sw128(sdO + off, 16, 1024),
-                 kIdescS, kk > 0);
+          for (int kk = 0; kk < D / 16; ++kk) {
+            const uint32_t off = ((kk / 4) * L::kBoxBytes + (kk % 4) * 32) >> 4;
+            mma_ss(tdP, desc_from_lo(v_lo + off), desc_from_lo(do_lo + off), kIdescS, kk > 0);
+          }
+          mma_commit(bar(kvDpFull));
         }
-        mma_commit(bar(kvDpFull));
+        __syncwarp();
       };
       for (int r = 0;; ++r, ++uc) {
         const int u = snake_unit(r, cta, n_cta);
@@ -229,15 +237,20 @@ attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         issue_dp(gs & 1);
         for (int s = 0; s < n_steps; ++s, ++gs) {
           const int st = gs & 1;
-          const uint32_t sQ = sbase + L::kQ0 + st * L::kStageBytes, sdO = sQ + L::kTileBytes;
+          const uint32_t stage = sbase + L::kQ0 + st * L::kStageBytes;
+          const uint32_t qT_lo = desc_lo(stage, L::kBoxBytes);                      // Q, MN-major
+          const uint32_t doT_lo = desc_lo(stage + L::kTileBytes, L::kBoxBytes);     // dO, MN-major
           const uint32_t acc = s > 0 ? 1u : 0u;
           mbar_wait(bar(kvPReady), gs & 1, s_abort);
           if (s == 0 && uc > 0) mbar_wait(bar(kvDkvRead), (uc - 1) & 1, s_abort);
           tc_fence_after();
+          if (leader) {
 #pragma unroll
-          for (int kk = 0; kk < kBM / 16; ++kk)   // dV += P^T dO
-            mma_ts(tdV, tS + kk * 8, smem_desc_sw128(sdO + kk * 2048, L::kBoxBytes, 1024), kIdescKV,
-                   acc | (kk > 0));
+            for (int kk = 0; kk < kBM / 16; ++kk)   // dV += P^T dO
+              mma_ts(tdV, tS + kk * 8, desc_from_lo(doT_lo + ((kk * 2048) >> 4)), kIdescKV,
+                     acc | (kk > 0));
+          }
+          __syncwarp();
           const bool more = (s + 1 < n_steps);
           const int g1 = gs + 1;
           if (more) {                              // S(s+1): P(s) was consumed by dV(s) above
@@ -247,24 +260,29 @@ attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           }
           mbar_wait(bar(kvDsReady), gs & 1, s_abort);
           tc_fence_after();
+          if (leader) {
 #pragma unroll
-          for (int kk = 0; kk < kBM / 16; ++kk) {   // dK += dS^T Q
-            const uint32_t off = (kk / 4) * L::kBoxBytes + (kk % 4) * 32;
-            mma_ss(tdK, smem_desc_sw128(sdS + off, 16, 1024),
-                   smem_desc_sw128(sQ + kk * 2048, L::kBoxBytes, 1024), kIdescKV, acc | (kk > 0));
+            for (int kk = 0; kk < kBM / 16; ++kk) {   // dK += dS^T Q
+              const uint32_t off = ((kk / 4) * L::kBoxBytes + (kk % 4) * 32) >> 4;
+              mma_ss(tdK, desc_from_lo(ds_lo + off), desc_from_lo(qT_lo + ((kk * 2048) >> 4)),
+                     kIdescKV, acc | (kk > 0));
+            }
+            mma_commit(bar(kvQdoEmpty0 + st));
           }
-          mma_commit(bar(kvQdoEmpty0 + st));
+          __syncwarp();
           if (more) {                              // dP(s+1): dP(s) was read before dS(s) was signalled
             mbar_wait(bar(kvDoFull0 + (g1 & 1)), (g1 >> 1) & 1, s_abort);
             tc_fence_after();
             issue_dp(g1 & 1);
           }
         }
-        mma_commit(bar(kvUnitDone));
-        mma_commit(bar(kvKvEmpty));
+        if (leader) {
+          mma_commit(bar(kvUnitDone));
+          mma_commit(bar(kvKvEmpty));
+        }
+        __syncwarp();
       }
     }
-    __syncwarp();
   } else {
     // =============================== compute ===============================================
     const int row = tid & 127;              // key row inside the block
@@ -418,11 +436,15 @@ struct DqSmem {
 };
 
 enum DqBar {
-  dqQFull = 0, dqQEmpty, dqKFull0, dqKFull1, dqKFull2, dqKEmpty0, dqKEmpty1, dqKEmpty2, dqVFull0,
-  dqVFull1, dqVEmpty0, dqVEmpty1, dqSFull0, dqSFull1, dqDpFull, dqDsReady, dqDone, dqRead,
+  dqQFull = 0, dqQEmpty, dqQtReady, dqKFull0, dqKFull1, dqKFull2, dqKEmpty0, dqKEmpty1, dqKEmpty2,
+  dqVFull0, dqVFull1, dqVEmpty0, dqVEmpty1, dqSFull, dqSRead, dqDpFull, dqDsReady, dqDone, dqRead,
   dqNumBars
 };
 
+// The query-side tiles Q and dO are the stationary A operands of S = Q K^T and dP = dO V^T.
+// They are copied once per unit from shared memory into tensor memory, so that those two
+// contractions read only K / V from shared memory (the shared-memory port, not the tensor
+// pipe, was the bound when all four operands came from there).
 template <int D, typename GradT>
 __global__ void __launch_bounds__(kWsThreads, 1)
 attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
@@ -433,7 +455,6 @@ attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
   using L = DqSmem<D>;
   extern __shared__ __align__(1024) uint8_t smem[];
   const uint32_t sbase = smem_u32(smem);
-  const uint32_t sQ = sbase + L::kQ, sdO = sbase + L::kdO;
   const uint32_t bars = sbase + L::kBars;
   auto bar = [&](int i) { return bars + 8u * (uint32_t)i; };
   volatile int* s_tmem = reinterpret_cast<volatile int*>(smem + L::kMisc);
@@ -443,10 +464,11 @@ attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
 
   if (tid == 0) {
     mbar_init(bar(dqQFull), 1);
-    mbar_init(bar(dqQEmpty), 1);
+    mbar_init(bar(dqQEmpty), kComputeThreads);
+    mbar_init(bar(dqQtReady), kComputeThreads);
     for (int i = dqKFull0; i <= dqVEmpty1; ++i) mbar_init(bar(i), 1);
-    mbar_init(bar(dqSFull0), 1);
-    mbar_init(bar(dqSFull1), 1);
+    mbar_init(bar(dqSFull), 1);
+    mbar_init(bar(dqSRead), kComputeThreads);
     mbar_init(bar(dqDpFull), 1);
     mbar_init(bar(dqDsReady), kComputeThreads);
     mbar_init(bar(dqDone), 1);
@@ -462,9 +484,10 @@ attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = static_cast<uint32_t>(*s_tmem);
-  // [0,128) S buffer 0, [128,256) S buffer 1, [256,384) dP (dS as bf16 reuses its first 64
-  // columns), [384, 384+D) dQ
-  const uint32_t tdP = tmem + 256, tdQ = tmem + 384;
+  // [0,128) S, [128,256) dP (dS as bf16 reuses its first 64 columns), [256,256+D) dQ,
+  // [384,384+D/2) Q as bf16 pairs, then D/2 columns of dO
+  const uint32_t tS = tmem, tdP = tmem + 128, tdQ = tmem + 256, tQ = tmem + 384,
+                 tdO = tmem + 384 + D / 2;
 
   const int G = Hq / Hkv;
   const bool plan_ok = (hdr[PK_HDR_PLAN_T] == T);
@@ -490,8 +513,8 @@ attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         mbar_expect_tx(bar(dqQFull), 2 * L::kTileBytes);
 #pragma unroll
         for (int b = 0; b < L::kBoxes; ++b) {
-          tma_load_2d(sQ + b * L::kBoxBytes, &tm_q, h * D + b * 64, q_start, bar(dqQFull));
-          tma_load_2d(sdO + b * L::kBoxBytes, &tm_do, h * D + b * 64, q_start, bar(dqQFull));
+          tma_load_2d(sbase + L::kQ + b * L::kBoxBytes, &tm_q, h * D + b * 64, q_start, bar(dqQFull));
+          tma_load_2d(sbase + L::kdO + b * L::kBoxBytes, &tm_do, h * D + b * 64, q_start, bar(dqQFull));
         }
         for (int j = 0; j < n_kv; ++j, ++gk) {
           const int ks = gk % L::kKStages, vs = gk % L::kVStages;
@@ -515,67 +538,79 @@ attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
     __syncwarp();
   } else if (warp == kMmaWarp) {
     // =============================== MMA issuer ===========================================
-    if (lane == 0) {
+    // The whole warp walks the schedule (so that addresses and descriptors stay warp-uniform);
+    // one elected lane issues the tensor-core instructions.
+    {
       constexpr uint32_t kIdescS = make_idesc(128, 128, kFmtBF16, kFmtBF16, 0, 0);
       constexpr uint32_t kIdescDQ = make_idesc(128, D, kFmtBF16, kFmtBF16, 0, 1);
+      const bool leader = elect_one();
       int gk = 0, uc = 0;
-      auto issue_s = [&](int g_idx) {       // S = Q K^T into S buffer (g_idx & 1)
+      auto issue_s = [&](int g_idx) {       // S = Q K^T, Q from tensor memory
         const int ks = g_idx % L::kKStages;
-        const uint32_t sK = sbase + L::kK0 + ks * L::kTileBytes;
-        const uint32_t tS = tmem + (g_idx & 1) * 128;
+        const uint32_t k_lo = desc_lo(sbase + L::kK0 + ks * L::kTileBytes, 16);
         mbar_wait(bar(dqKFull0 + ks), (g_idx / L::kKStages) & 1, s_abort);
         tc_fence_after();
+        if (leader) {
 #pragma unroll
-        for (int kk = 0; kk < D / 16; ++kk) {
-          const uint32_t off = (kk / 4) * L::kBoxBytes + (kk % 4) * 32;
-          mma_ss(tS, smem_desc_sw128(sQ + off, 16, 1024), smem_desc_sw128(sK + off, 16, 1024),
-                 kIdescS, kk > 0);
+          for (int kk = 0; kk < D / 16; ++kk) {
+            const uint32_t off = (kk / 4) * L::kBoxBytes + (kk % 4) * 32;
+            mma_ts(tS, tQ + kk * 8, desc_from_lo(k_lo + (off >> 4)), kIdescS, kk > 0);
+          }
+          mma_commit(bar(dqSFull));
         }
-        mma_commit(bar(dqSFull0 + (g_idx & 1)));
+        __syncwarp();
       };
       auto issue_dp = [&](int g_idx) {      // dP = dO V^T; the V stage is free once it completes
         const int vs = g_idx % L::kVStages;
-        const uint32_t sV = sbase + L::kV0 + vs * L::kTileBytes;
+        const uint32_t v_lo = desc_lo(sbase + L::kV0 + vs * L::kTileBytes, 16);
         mbar_wait(bar(dqVFull0 + vs), (g_idx / L::kVStages) & 1, s_abort);
         tc_fence_after();
+        if (leader) {
 #pragma unroll
-        for (int kk = 0; kk < D / 16; ++kk) {
-          const uint32_t off = (kk / 4) * L::kBoxBytes + (kk % 4) * 32;
-          mma_ss(tdP, smem_desc_sw128(sdO + off, 16, 1024), smem_desc_sw128(sV + off, 16, 1024),
-                 kIdescS, kk > 0);
+          for (int kk = 0; kk < D / 16; ++kk) {
+            const uint32_t off = (kk / 4) * L::kBoxBytes + (kk % 4) * 32;
+            mma_ts(tdP, tdO + kk * 8, desc_from_lo(v_lo + (off >> 4)), kIdescS, kk > 0);
+          }
+          mma_commit(bar(dqDpFull));
+          mma_commit(bar(dqVEmpty0 + vs));
         }
-        mma_commit(bar(dqDpFull));
-        mma_commit(bar(dqVEmpty0 + vs));
+        __syncwarp();
       };
       for (int r = 0;; ++r, ++uc) {
         const int u = snake_unit(r, cta, n_cta);
         if (u >= n_units || *s_abort) break;
         const int4 it = items[order[u / Hq]];
         const int n_kv = (it.w + kBN - 1) / kBN;
-        mbar_wait(bar(dqQFull), uc & 1, s_abort);
+        mbar_wait(bar(dqQtReady), uc & 1, s_abort);
+        if (gk > 0) mbar_wait(bar(dqSRead), (gk - 1) & 1, s_abort);   // S of the previous step read
         tc_fence_after();
         issue_s(gk);
         issue_dp(gk);
         for (int j = 0; j < n_kv; ++j, ++gk) {
           const int ks = gk % L::kKStages;
-          const uint32_t sK = sbase + L::kK0 + ks * L::kTileBytes;
+          const uint32_t k_lo = desc_lo(sbase + L::kK0 + ks * L::kTileBytes, L::kBoxBytes);
           const bool more = (j + 1 < n_kv);
-          if (more) issue_s(gk + 1);   // other S buffer: its last reader signalled dS(j-1) already
+          if (more) {   // the single S buffer is free as soon as the compute warps have loaded S(j)
+            mbar_wait(bar(dqSRead), gk & 1, s_abort);
+            issue_s(gk + 1);
+          }
           mbar_wait(bar(dqDsReady), gk & 1, s_abort);
           if (j == 0 && uc > 0) mbar_wait(bar(dqRead), (uc - 1) & 1, s_abort);
           tc_fence_after();
+          if (leader) {
 #pragma unroll
-          for (int kk = 0; kk < kBN / 16; ++kk)   // dQ += dS K   (dS from tensor memory)
-            mma_ts(tdQ, tdP + kk * 8, smem_desc_sw128(sK + kk * 2048, L::kBoxBytes, 1024), kIdescDQ,
-                   (j > 0) | (kk > 0));
-          mma_commit(bar(dqKEmpty0 + ks));
+            for (int kk = 0; kk < kBN / 16; ++kk)   // dQ += dS K   (dS from tensor memory)
+              mma_ts(tdQ, tdP + kk * 8, desc_from_lo(k_lo + ((kk * 2048) >> 4)), kIdescDQ,
+                     (j > 0) | (kk > 0));
+            mma_commit(bar(dqKEmpty0 + ks));
+          }
+          __syncwarp();
           if (more) issue_dp(gk + 1);   // overwrites dP/dS(j) after dQ(j) (same pipe, in order)
         }
-        mma_commit(bar(dqDone));
-        mma_commit(bar(dqQEmpty));
+        if (leader) mma_commit(bar(dqDone));
+        __syncwarp();
       }
     }
-    __syncwarp();
   } else {
     // =============================== compute ===============================================
     const int row = tid & 127;              // query row inside the tile
@@ -592,9 +627,33 @@ attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
       const int tok = q_start + row;
       const float lse2 = (tok < T) ? lse[(size_t)h * T + tok] * kLog2eWs : 0.f;
       const float dl = (tok < T) ? delta[(size_t)h * T + tok] : 0.f;
+
+      // ---- Q and dO rows: shared memory (128B-swizzled) -> tensor memory, half a row per thread
+      mbar_wait(bar(dqQFull), uc & 1, s_abort);
+      if (qd < 2) {
+        constexpr int kElems = D / 2;                       // elements per thread
+        const int box = (qd * kElems) / 64, chunk0 = ((qd * kElems) % 64) / 8;
+#pragma unroll
+        for (int which = 0; which < 2; ++which) {
+          const uint8_t* src = smem + (which == 0 ? L::kQ : L::kdO) + box * L::kBoxBytes + row * 128;
+          uint32_t v[kElems / 2];
+#pragma unroll
+          for (int c = 0; c < kElems / 8; ++c) {
+            const uint4 x = *reinterpret_cast<const uint4*>(src + (((chunk0 + c) ^ (row & 7)) << 4));
+            v[4 * c] = x.x; v[4 * c + 1] = x.y; v[4 * c + 2] = x.z; v[4 * c + 3] = x.w;
+          }
+          const uint32_t dst = (which == 0 ? tQ : tdO) + lane_off + qd * (kElems / 2);
+          if (kElems == 64) tmem_st32(dst, v);
+          else tmem_st16(dst, v);
+        }
+        tmem_wait_st();
+      }
+      tc_fence_before();
+      mbar_arrive(bar(dqQtReady));
+      mbar_arrive(bar(dqQEmpty));      // the shared-memory copies may be overwritten
+
       for (int j = 0; j < n_kv; ++j, ++gk) {
-        const uint32_t tS = tmem + (gk & 1) * 128;
-        mbar_wait(bar(dqSFull0 + (gk & 1)), (gk >> 1) & 1, s_abort);
+        mbar_wait(bar(dqSFull), gk & 1, s_abort);
         tc_fence_after();
         float p[kCW];
         {
@@ -602,6 +661,8 @@ attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
 #pragma unroll
           for (int c0 = 0; c0 < kCW; c0 += 32) tmem_ld32(tS + lane_off + qd * kCW + c0, sv + c0);
           tmem_wait_ld();
+          tc_fence_before();
+          mbar_arrive(bar(dqSRead));
 #pragma unroll
           for (int c = 0; c < kCW; ++c)
             p[c] = fast_exp2(fmaf(__uint_as_float(sv[c]), scale_log2, -lse2));

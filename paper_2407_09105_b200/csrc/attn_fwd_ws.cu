@@ -151,20 +151,26 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
     __syncwarp();
   } else if (warp == kFwsMmaWarp) {
     // =============================== MMA issuer ===========================================
-    if (lane == 0) {
+    // The whole warp walks the schedule (so that addresses and descriptors stay warp-uniform);
+    // one elected lane issues the tensor-core instructions.
+    {
       constexpr uint32_t kIdescQK = make_idesc(128, 128, kFmtBF16, kFmtBF16, 0, 0);
       constexpr uint32_t kIdescPV = make_idesc(128, D, kFmtBF16, kFmtBF16, 0, 1);
+      const bool leader = elect_one();
       int gk = 0, uc = 0;
       auto issue_s = [&](int t, int st) {
-        const uint32_t sQ = sbase + L::kQ0 + t * L::kTileBytes;
-        const uint32_t sK = sbase + L::kKV0 + st * L::kStageBytes;
+        const uint32_t q_lo = desc_lo(sbase + L::kQ0 + t * L::kTileBytes, 16);
+        const uint32_t k_lo = desc_lo(sbase + L::kKV0 + st * L::kStageBytes, 16);
+        if (leader) {
 #pragma unroll
-        for (int kk = 0; kk < D / 16; ++kk) {
-          const uint32_t off = (kk / 4) * L::kBoxBytes + (kk % 4) * 32;
-          mma_ss(tmem + t * 128, smem_desc_sw128(sQ + off, 16, 1024),
-                 smem_desc_sw128(sK + off, 16, 1024), kIdescQK, kk > 0);
+          for (int kk = 0; kk < D / 16; ++kk) {
+            const uint32_t off = ((kk / 4) * L::kBoxBytes + (kk % 4) * 32) >> 4;
+            mma_ss(tmem + t * 128, desc_from_lo(q_lo + off), desc_from_lo(k_lo + off), kIdescQK,
+                   kk > 0);
+          }
+          mma_commit(bar(fSFull0 + t));
         }
-        mma_commit(bar(fSFull0 + t));
+        __syncwarp();
       };
       for (int r = 0;; ++r, ++uc) {
         const int u = snake_unit_f(r, cta, n_cta);
@@ -178,20 +184,23 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         issue_s(1, gk & 1);
         for (int j = 0; j < n_kv; ++j, ++gk) {
           const int st = gk & 1;
-          const uint32_t sV = sbase + L::kKV0 + st * L::kStageBytes + L::kTileBytes;
+          const uint32_t v_lo =
+              desc_lo(sbase + L::kKV0 + st * L::kStageBytes + L::kTileBytes, L::kBoxBytes);
           const bool more = (j + 1 < n_kv);
 #pragma unroll
           for (int t = 0; t < 2; ++t) {
             mbar_wait(bar(fPReady0 + t), gk & 1, s_abort);
             if (j == 0 && uc > 0) mbar_wait(bar(fORead0 + t), (uc - 1) & 1, s_abort);
             tc_fence_after();
+            if (leader) {
 #pragma unroll
-            for (int kk = 0; kk < kBN / 16; ++kk)   // O_t += P_t V
-              mma_ts(tmem + 256 + t * 128, tmem + t * 128 + kk * 8,
-                     smem_desc_sw128(sV + kk * 2048, L::kBoxBytes, 1024), kIdescPV,
-                     (j > 0) | (kk > 0));
-            if (t == 1) mma_commit(bar(fKvEmpty0 + st));
-            if (!more) mma_commit(bar(fOFull0 + t));
+              for (int kk = 0; kk < kBN / 16; ++kk)   // O_t += P_t V
+                mma_ts(tmem + 256 + t * 128, tmem + t * 128 + kk * 8,
+                       desc_from_lo(v_lo + ((kk * 2048) >> 4)), kIdescPV, (j > 0) | (kk > 0));
+              if (t == 1) mma_commit(bar(fKvEmpty0 + st));
+              if (!more) mma_commit(bar(fOFull0 + t));
+            }
+            __syncwarp();
             if (more) {                              // S_t(j+1): P_t(j) was consumed just above
               if (t == 0) {
                 mbar_wait(bar(fKvFull0 + ((gk + 1) & 1)), ((gk + 1) >> 1) & 1, s_abort);
@@ -201,10 +210,10 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             }
           }
         }
-        mma_commit(bar(fQEmpty));
+        if (leader) mma_commit(bar(fQEmpty));
+        __syncwarp();
       }
     }
-    __syncwarp();
   } else {
     // =============================== softmax (warps 0-3: tile 0, warps 4-7: tile 1) =======
     const int t = tid >> 7;

@@ -163,6 +163,17 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr, uint32_t lbo
   return d;
 }
 
+// The same descriptor split in two 32-bit halves, so that an issue loop only adds a constant to
+// the low half: high = stride offset 1024 B, version, 128-byte swizzle (fixed for every tile
+// here); low = start address and the leading offset.
+constexpr uint32_t kDescHiSw128 = (1024u >> 4) | (1u << 14) | (2u << 29);
+__device__ __forceinline__ uint32_t desc_lo(uint32_t saddr, uint32_t lbo_bytes) {
+  return ((saddr & 0x3FFFFu) >> 4) | (((lbo_bytes >> 4) & 0x3FFFu) << 16);
+}
+__device__ __forceinline__ uint64_t desc_from_lo(uint32_t lo) {
+  return (static_cast<uint64_t>(kDescHiSw128) << 32) | lo;
+}
+
 // Instruction descriptor of kind::f16: 16-bit A and B, fp32 accumulator, dense.  A and B
 // must have the SAME format (both fp16 or both bf16): a mixed pair is rejected by the
 // hardware as an illegal instruction.
