@@ -15,10 +15,10 @@
 // Both recompute S and dP (7 contractions per tile pair instead of 5), both are bitwise
 // reproducible, and both never visit a tile outside an example's causal block.
 //
-// Roles: 16 compute warps (lane = tensor-memory row; warp w works on columns
-// [32*(w/4), 32*(w/4)+32) of the rows of lane quarter w%4 -- many warps, because the compute
-// phases are bound by latency, not by issue or special-function throughput), one warp that
-// issues every tcgen05.mma, one warp that drives TMA.
+// Roles: 8 compute warps (lane = tensor-memory row; warp w works on columns [64*(w/4), +64) of
+// the rows of lane quarter w%4; 16 warps of 32 columns measured slightly slower because they
+// take issue slots from the warp that feeds the tensor pipe), one warp that walks the MMA
+// schedule with one elected lane issuing every tcgen05.mma, one warp that drives TMA.
 // Units are assigned statically: CTA c takes positions c, 2P-1-c, 2P+c, ... of the plan's
 // longest-first order, so the roles enumerate the same sequence without talking to each other.
 // Every wait is bounded; on expiry an abort flag makes all later waits return at once.
@@ -35,7 +35,7 @@ namespace {
 using namespace ptx;
 
 #ifndef PK_BWD_COMPUTE_THREADS
-#define PK_BWD_COMPUTE_THREADS 512
+#define PK_BWD_COMPUTE_THREADS 256
 #endif
 constexpr int kComputeThreads = PK_BWD_COMPUTE_THREADS;   // 256 or 512
 constexpr int kNQ = kComputeThreads / 128;                // column groups per tile row
