@@ -43,6 +43,7 @@ constexpr int kCW = 128 / kNQ;                            // columns per compute
 constexpr int kWsThreads = kComputeThreads + 64;
 constexpr int kMmaWarp = kComputeThreads / 32;
 constexpr int kLoadWarp = kMmaWarp + 1;
+static_assert(kNQ == 2, "the dK/dV kernel assigns two 32-column pieces per compute thread");
 constexpr float kLog2eWs = 1.4426950408889634f;
 
 // position in the longest-first order of the r-th unit of this CTA (snake over the rounds)
@@ -75,7 +76,7 @@ struct DkvSmem {
 
 enum DkvBar {
   kvKvFull = 0, kvKvEmpty, kvQFull0, kvQFull1, kvDoFull0, kvDoFull1, kvQdoEmpty0, kvQdoEmpty1,
-  kvSFull, kvDpFull, kvPReady, kvDsReady, kvUnitDone, kvDkvRead, kvNumBars
+  kvSFull, kvDpFull, kvPReady, kvPReadyA, kvDsReady, kvUnitDone, kvDkvRead, kvNumBars
 };
 
 template <int D, typename GradT>
@@ -111,6 +112,7 @@ attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     mbar_init(bar(kvSFull), 1);
     mbar_init(bar(kvDpFull), 1);
     mbar_init(bar(kvPReady), kComputeThreads);
+    mbar_init(bar(kvPReadyA), kComputeThreads);
     mbar_init(bar(kvDsReady), kComputeThreads);
     mbar_init(bar(kvUnitDone), 1);
     mbar_init(bar(kvDkvRead), kComputeThreads);
@@ -241,14 +243,22 @@ attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           const uint32_t qT_lo = desc_lo(stage, L::kBoxBytes);                      // Q, MN-major
           const uint32_t doT_lo = desc_lo(stage + L::kTileBytes, L::kBoxBytes);     // dO, MN-major
           const uint32_t acc = s > 0 ? 1u : 0u;
-          mbar_wait(bar(kvPReady), gs & 1, s_abort);
+          mbar_wait(bar(kvPReadyA), gs & 1, s_abort);   // first 64 query columns of P
           if (s == 0 && uc > 0) mbar_wait(bar(kvDkvRead), (uc - 1) & 1, s_abort);
           tc_fence_after();
           if (leader) {
 #pragma unroll
-            for (int kk = 0; kk < kBM / 16; ++kk)   // dV += P^T dO
+            for (int kk = 0; kk < kBM / 32; ++kk)   // dV += P^T dO, first half of the query rows
               mma_ts(tdV, tS + kk * 8, desc_from_lo(doT_lo + ((kk * 2048) >> 4)), kIdescKV,
                      acc | (kk > 0));
+          }
+          __syncwarp();
+          mbar_wait(bar(kvPReady), gs & 1, s_abort);    // second half
+          tc_fence_after();
+          if (leader) {
+#pragma unroll
+            for (int kk = kBM / 32; kk < kBM / 16; ++kk)
+              mma_ts(tdV, tS + kk * 8, desc_from_lo(doT_lo + ((kk * 2048) >> 4)), kIdescKV, 1u);
           }
           __syncwarp();
           const bool more = (s + 1 < n_steps);
@@ -301,64 +311,67 @@ attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           const int st = gs & 1;
           const int q_left = q_len - i * kBM;
           const int col_min = (i == 0) ? row : 0;
-          const float4* lse4 = reinterpret_cast<const float4*>(s_lse + st * 128 + qd * kCW);
-          const float4* dl4 = reinterpret_cast<const float4*>(s_delta + st * 128 + qd * kCW);
+          // This thread's 64 query columns are taken in two pieces, [32*qd, +32) of the first 64
+          // and of the second 64, so that all warps finish the first half of P together and dV
+          // can start on it while the second half is still being exponentiated.
+          const int col_a = qd * 32, col_b = 64 + qd * 32;
           mbar_wait(bar(kvQFull0 + st), (gs >> 1) & 1, s_abort);   // lse / delta rows visible
           mbar_wait(bar(kvSFull), gs & 1, s_abort);
           tc_fence_after();
-          float p[kCW];
-          {
-            uint32_t sv[kCW];
+          float p[64];
+          uint32_t sv[64];
+          tmem_ld32(tS + lane_off + col_a, sv);
+          tmem_ld32(tS + lane_off + col_b, sv + 32);
+          tmem_wait_ld();
+          const bool edge = (i == 0 || q_left < kBM);   // diagonal tile or last, partial tile
 #pragma unroll
-            for (int c0 = 0; c0 < kCW; c0 += 32) tmem_ld32(tS + lane_off + qd * kCW + c0, sv + c0);
-            tmem_wait_ld();
+          for (int half = 0; half < 2; ++half) {
+            const int col0 = half == 0 ? col_a : col_b;
+            const float4* lse4 = reinterpret_cast<const float4*>(s_lse + st * 128 + col0);
 #pragma unroll
-            for (int c = 0; c < kCW; c += 4) {
+            for (int c = 0; c < 32; c += 4) {
               const float4 l4 = lse4[c >> 2];
-              p[c] = fast_exp2(fmaf(__uint_as_float(sv[c]), scale_log2, -l4.x));
-              p[c + 1] = fast_exp2(fmaf(__uint_as_float(sv[c + 1]), scale_log2, -l4.y));
-              p[c + 2] = fast_exp2(fmaf(__uint_as_float(sv[c + 2]), scale_log2, -l4.z));
-              p[c + 3] = fast_exp2(fmaf(__uint_as_float(sv[c + 3]), scale_log2, -l4.w));
+              const int k = half * 32 + c;
+              p[k] = fast_exp2(fmaf(__uint_as_float(sv[k]), scale_log2, -l4.x));
+              p[k + 1] = fast_exp2(fmaf(__uint_as_float(sv[k + 1]), scale_log2, -l4.y));
+              p[k + 2] = fast_exp2(fmaf(__uint_as_float(sv[k + 2]), scale_log2, -l4.z));
+              p[k + 3] = fast_exp2(fmaf(__uint_as_float(sv[k + 3]), scale_log2, -l4.w));
             }
-            // masks are needed only on the diagonal tile (causal) and on a last, partial tile
-            // (query rows past the example end); interior tiles skip the compares
-            if (i == 0 || q_left < kBM) {
+            if (edge) {   // interior tiles skip the compares
 #pragma unroll
-              for (int c = 0; c < kCW; ++c) {
-                const int col = qd * kCW + c;
-                if (!((col >= col_min) && (col < q_left))) p[c] = 0.f;
+              for (int c = 0; c < 32; ++c) {
+                const int col = col0 + c;
+                if (!((col >= col_min) && (col < q_left))) p[half * 32 + c] = 0.f;
               }
             }
-          }
-          // every column group must have read S before P overwrites its columns
-          tc_fence_before();
-          compute_bar_sync();
-          tc_fence_after();
-          {
-            uint32_t pp[kCW / 2];
+            if (half == 0) {   // every thread has loaded S: P may overwrite its columns
+              tc_fence_before();
+              compute_bar_sync();
+              tc_fence_after();
+            }
+            uint32_t pp[16];
 #pragma unroll
-            for (int c = 0; c < kCW / 2; ++c) pp[c] = pack_bf16x2(p[2 * c], p[2 * c + 1]);
-            if (kCW == 64) tmem_st32(tS + lane_off + qd * (kCW / 2), pp);
-            else tmem_st16(tS + lane_off + qd * (kCW / 2), pp);
+            for (int c = 0; c < 16; ++c) pp[c] = pack_bf16x2(p[half * 32 + 2 * c], p[half * 32 + 2 * c + 1]);
+            tmem_st16(tS + lane_off + half * 32 + qd * 16, pp);
             tmem_wait_st();
+            tc_fence_before();
+            mbar_arrive(bar(half == 0 ? kvPReadyA : kvPReady));
           }
-          tc_fence_before();
-          mbar_arrive(bar(kvPReady));
 
           mbar_wait(bar(kvDpFull), gs & 1, s_abort);
           tc_fence_after();
-          // dS^T row `row`, query columns [qd*kCW, +kCW): box (qd*kCW)/64, 16-byte chunks from
-          // ((qd*kCW)%64)/8 on
-          uint8_t* ds_row = smem + L::kdS + ((qd * kCW) / 64) * L::kBoxBytes + row * 128;
-          constexpr int kChunk0 = 0;
 #pragma unroll
-          for (int c2 = 0; c2 < kCW / 32; ++c2) {
+          for (int c2 = 0; c2 < 2; ++c2) {
+            const int col0 = c2 == 0 ? col_a : col_b;
+            // dS^T row `row`, query columns [col0, +32): box c2, 16-byte chunks 4*qd .. 4*qd+3
+            uint8_t* ds_row = smem + L::kdS + c2 * L::kBoxBytes + row * 128;
+            const float4* dl4 = reinterpret_cast<const float4*>(s_delta + st * 128 + col0);
             uint32_t dp[32], dd[16];
-            tmem_ld32(tdP + lane_off + qd * kCW + c2 * 32, dp);
+            tmem_ld32(tdP + lane_off + col0, dp);
             tmem_wait_ld();
 #pragma unroll
             for (int e = 0; e < 32; e += 4) {
-              const float4 d4 = dl4[(c2 * 32 + e) >> 2];
+              const float4 d4 = dl4[e >> 2];
               const float d0 = p[c2 * 32 + e] * (__uint_as_float(dp[e]) - d4.x);
               const float d1 = p[c2 * 32 + e + 1] * (__uint_as_float(dp[e + 1]) - d4.y);
               const float d2 = p[c2 * 32 + e + 2] * (__uint_as_float(dp[e + 2]) - d4.z);
@@ -366,10 +379,9 @@ attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
               dd[e >> 1] = pack_bf16x2(d0, d1);
               dd[(e >> 1) + 1] = pack_bf16x2(d2, d3);
             }
-            const int chunk_base = kChunk0 + ((qd * kCW) % 64) / 8 + c2 * 4;
 #pragma unroll
             for (int ch = 0; ch < 4; ++ch) {
-              const int chunk = (chunk_base + ch) ^ (row & 7);
+              const int chunk = (qd * 4 + ch) ^ (row & 7);
               *reinterpret_cast<uint4*>(ds_row + (chunk << 4)) =
                   make_uint4(dd[ch * 4], dd[ch * 4 + 1], dd[ch * 4 + 2], dd[ch * 4 + 3]);
             }
