@@ -35,9 +35,9 @@ from paper_2407_09105_b200 import workloads as wl  # noqa: E402
 METRIC = "packed_attn_fwd_bwd_useful_tflops"
 UNIT = "TFLOP/s"
 
-# DRAM bytes per causal (query, key, q-head) pair of the backward main kernel, from the ncu
+# DRAM bytes per causal (query, key, q-head) pair of the dominant (dK/dV) kernel, from the ncu
 # capture summarised in profiles/ (scaled to a launch by the number of pairs); None = not captured.
-NCU_BWD_DRAM_BYTES_PER_PAIR = None
+NCU_BWD_DRAM_BYTES_PER_PAIR = 0.5778   # attn_bwd_dkv_kernel, profiles/attn_kernels_c4_2packs.txt
 
 
 def _peaks():
@@ -316,7 +316,7 @@ def main():
         "kernel": "attn_bwd_dkv_kernel" if split else "attn_bwd_kernel", "bound": "tensor", "achieved": bwd_tflops,
         "peak": peaks["sustained"], "peak_kind": f"bf16 sustained, {peaks['source']}",
         "peak_burst": peaks["burst"], "unit": "TFLOP/s", "frac": bwd_tflops / peaks["sustained"],
-        "traffic": (None if NCU_BWD_DRAM_BYTES_PER_PAIR is None
+        "traffic": (None if (NCU_BWD_DRAM_BYTES_PER_PAIR is None or not split)
                     else NCU_BWD_DRAM_BYTES_PER_PAIR * w.causal_pairs * Hq),
         "ms_per_launch": bwd_ms,
         "note": ("dK/dV kernel: useful = dV and dK (4*D FLOPs per causal pair and head); it also "
