@@ -181,6 +181,8 @@ def main():
     ap.add_argument("--impl", default="ours")
     ap.add_argument("--packs", type=int, default=0,
                     help="use only the first N packs of the workload (small cases for profiling)")
+    ap.add_argument("--per-stream", action="store_true",
+                    help="one call per pack / mini-batch instead of one flat stream")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -214,17 +216,39 @@ def main():
     T, Hq, D = st.q.shape
     Hkv = st.k.shape[1]
     scale, theta = w.softmax_scale, w.rope_theta
-    ws = api.alloc_workspace(T, Hq, Hkv, D)
     out = torch.empty_like(st.q)
     lse = torch.empty((Hq, T), dtype=torch.float32, device="cuda")
     dq, dk, dv = torch.empty_like(st.q), torch.empty_like(st.k), torch.empty_like(st.v)
     stream = torch.cuda.current_stream()
 
-    def step():
-        api.pk_attn_fwd(st.q, st.k, st.v, st.position_ids, scale, theta, out, lse, ws,
-                        reuse_plan=False, stream=stream)
-        api.pk_attn_bwd(st.dout, st.q, st.k, st.v, out, lse, st.position_ids, scale, theta,
-                        dq, dk, dv, ws, reuse_plan=True, stream=stream)
+    if args.per_stream:
+        # one call per packed stream (mini-batch / pack), all on the same CUDA stream: the same
+        # tokens as the flat run, cut at the stream edges
+        bounds = np.concatenate([[0], np.cumsum([sum(x) for x in w.streams])]).tolist()
+        ws = api.alloc_workspace(max(b - a for a, b in zip(bounds, bounds[1:])), Hq, Hkv, D)
+        pieces = []
+        for a, b in zip(bounds, bounds[1:]):
+            n = b - a
+            pieces.append((st.q[a:b], st.k[a:b], st.v[a:b], st.dout[a:b], st.position_ids[a:b],
+                           out[a:b], torch.empty((Hq, n), dtype=torch.float32, device="cuda"),
+                           dq[a:b], dk[a:b], dv[a:b]))
+
+        def step():
+            for (q_, k_, v_, do_, pos_, out_, lse_, dq_, dk_, dv_) in pieces:
+                api.pk_attn_fwd(q_, k_, v_, pos_, scale, theta, out_, lse_, ws,
+                                reuse_plan=False, stream=stream)
+                api.pk_attn_bwd(do_, q_, k_, v_, out_, lse_, pos_, scale, theta,
+                                dq_, dk_, dv_, ws, reuse_plan=True, stream=stream)
+        calls_per_step = len(pieces)
+    else:
+        ws = api.alloc_workspace(T, Hq, Hkv, D)
+
+        def step():
+            api.pk_attn_fwd(st.q, st.k, st.v, st.position_ids, scale, theta, out, lse, ws,
+                            reuse_plan=False, stream=stream)
+            api.pk_attn_bwd(st.dout, st.q, st.k, st.v, out, lse, st.position_ids, scale, theta,
+                            dq, dk, dv, ws, reuse_plan=True, stream=stream)
+        calls_per_step = 1
 
     def barrier():
         if dist is not None:
@@ -251,8 +275,9 @@ def main():
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record(stream)
     for i in range(args.steps):
-        for k, pairs in kev.items():
-            api.pk_set_timing_events(k, pairs[i][0], pairs[i][1])
+        if calls_per_step == 1:
+            for k, pairs in kev.items():
+                api.pk_set_timing_events(k, pairs[i][0], pairs[i][1])
         step()
     e1.record(stream)
     barrier()
@@ -304,6 +329,8 @@ def main():
         return
 
     peaks = _peaks()
+    if calls_per_step > 1:      # per-kernel events are recorded for the flat run only
+        fwd_ms = bwd_ms = dq_ms = float('nan')
     # without fused RoPE the backward is two kernels: dK/dV (6 of the 10 useful FLOPs per pair and
     # head-dim: dV, dK, plus one of the two recomputed products) and dQ.  The dominant kernel is
     # the dK/dV one; its useful work is dV and dK only: 4*D FLOPs per pair.
@@ -338,7 +365,8 @@ def main():
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": f"{w.name}: {w.packing}, {len(w.streams)} packs as one flat stream",
+        "config": {"workload": (f"{w.name}: {w.packing}, {len(w.streams)} packs, " +
+                                ("one call per pack" if args.per_stream else "as one flat stream")),
                    "tokens": T, "examples": len(lens), "Hq": Hq, "Hkv": Hkv, "head_dim": D,
                    "rope_theta": theta, "causal_pairs": w.causal_pairs,
                    "flop_convention": "14*D*Hq*sum L(L+1)/2", "l2": "inputs_exceed_l2",
@@ -347,8 +375,8 @@ def main():
         "pct_of_bf16_peak": {"sustained": 100 * value / world / peaks["sustained"],
                              "burst": 100 * value / world / peaks["burst"],
                              "source": peaks["source"]},
-        "clocks": clocks, "e2e": e2e, "gpu_launches": (5 + (2 if theta > 0 else 0)) * args.steps,
-        "roofline": roofline, "cpu_baseline": cpu_baseline,
+        "clocks": clocks, "e2e": e2e, "gpu_launches": (5 + (2 if theta > 0 else 0)) * args.steps * calls_per_step,
+        "roofline": roofline if calls_per_step == 1 else None, "cpu_baseline": cpu_baseline,
     }
     print(json.dumps(line))
     if dist is not None:
