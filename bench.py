@@ -106,6 +106,17 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
+def _launches_per_call(theta, Hq, Hkv, D):
+    """Kernels of this library per forward+backward pair (default RoPE mode)."""
+    if theta <= 0:
+        return 5                      # plan, forward, delta, dK/dV, dQ
+    pairs = (Hq // Hkv) % 2 == 0
+    if D == 128:                      # rotated fp16 copies of q and k
+        fwd = 4 if pairs else 3       # plan, rotate q, rotate k, forward | plan, table, forward
+        return fwd + 6                # table, delta, rotate q, rotate k, dK/dV, dQ
+    return 3 + 4                      # in-tile: plan, table, forward | table, delta, backward, dQ finish
+
+
 def _oracle_sample(w: wl.Workload):
     """A bounded sample of whole examples of the workload for the CPU oracle: the example
     closest to 2048 tokens plus the eight shortest ones, all heads."""
@@ -375,7 +386,7 @@ def main():
         "pct_of_bf16_peak": {"sustained": 100 * value / world / peaks["sustained"],
                              "burst": 100 * value / world / peaks["burst"],
                              "source": peaks["source"]},
-        "clocks": clocks, "e2e": e2e, "gpu_launches": (5 + (2 if theta > 0 else 0)) * args.steps * calls_per_step,
+        "clocks": clocks, "e2e": e2e, "gpu_launches": _launches_per_call(theta, Hq, Hkv, D) * args.steps * calls_per_step,
         "roofline": roofline if calls_per_step == 1 else None, "cpu_baseline": cpu_baseline,
     }
     print(json.dumps(line))

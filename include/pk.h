@@ -165,6 +165,20 @@ int pk_attn_bwd(const void* dout, const void* q, const void* k, const void* v,
 int pk_status_read(const void* workspace, void* stream, int32_t* code, int32_t* detail);
 
 /*
+ * How the attention calls apply RoPE when rope_theta > 0 (process-wide; the paper is silent on
+ * RoPE, both modes compute the same function):
+ *   PK_ROPE_ROTATED_COPIES (default)  one pass writes rotated fp16 copies of q and k into the
+ *       workspace (it reuses the PK_WS_DQ_ACC section), then the warp-specialised kernels run
+ *       on them and rotate dQ/dK back in their epilogues.  A K tile is visited by every query
+ *       tile of every head of its group, so rotating once costs one HBM pass instead of one
+ *       rotation per visit.  Needs D == 128 and an even Hq/Hkv; other shapes use the in-tile mode.
+ *   PK_ROPE_IN_TILE  the Q/K tiles are rotated in shared memory right after their TMA load.
+ */
+#define PK_ROPE_ROTATED_COPIES 0
+#define PK_ROPE_IN_TILE        1
+int pk_set_rope_mode(int32_t mode);
+
+/*
  * pk_seqlens_from_posids for callers that cannot give the library a workspace and for whom
  * a device allocation is not an option (the paper has no counterpart; it is the same
  * boundary recovery as pk_seqlens_from_posids with the same outputs).  Typical callers: a

@@ -49,6 +49,7 @@ _SIGNATURES = {
                                    _vp, _vp, _vp, _i32, _i32, _vp, _sz, _vp]),
     "pk_status_read": (ctypes.c_int, [_vp, _vp, ctypes.POINTER(_i32), ctypes.POINTER(_i32)]),
     "pk_set_timing_events": (ctypes.c_int, [_i32, _vp, _vp]),
+    "pk_set_rope_mode": (ctypes.c_int, [_i32]),
     "pk_seqlens_from_posids_noalloc": (ctypes.c_int, [_vp, _i32, _vp, _vp, _vp, _vp]),
 }
 
@@ -206,6 +207,13 @@ def pk_set_timing_events(which: int, start: Optional[torch.cuda.Event],
     s = None if start is None else start.cuda_event
     e = None if stop is None else stop.cuda_event
     _check("pk_set_timing_events", lib().pk_set_timing_events(which, s, e))
+
+
+PK_ROPE_ROTATED_COPIES, PK_ROPE_IN_TILE = 0, 1
+
+
+def pk_set_rope_mode(mode: int) -> None:
+    _check("pk_set_rope_mode", lib().pk_set_rope_mode(mode))
 
 
 def workspace_view(workspace: torch.Tensor, which: int, T: int, Hq: int, Hkv: int, D: int,

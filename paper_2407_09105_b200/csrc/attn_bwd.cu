@@ -498,6 +498,7 @@ extern "C" int pk_attn_bwd(const void* dout, const void* q, const void* k, const
     if (rc != PK_OK) return rc;
   }
   const bool use_rope = rope_theta > 0.f;
+  const bool rotated_copies = use_rope && g_rope_mode == PK_ROPE_ROTATED_COPIES && D == 128;
   float* table = reinterpret_cast<float*>(ws + lay.off[PK_WS_ROPE_TABLE]);
   if (use_rope) {
     rc = rope_table_launch(position_ids, T, D, rope_theta, table, stream);
@@ -520,8 +521,8 @@ extern "C" int pk_attn_bwd(const void* dout, const void* q, const void* k, const
       delta_kernel<float><<<blocks, warps * 32, 0, stream>>>(
           static_cast<const __nv_bfloat16*>(dout), static_cast<const float*>(out), delta, T, Hq, D);
     if ((rc = launch_status()) != PK_OK) return rc;
-    // only the fused-RoPE kernel accumulates dQ with reductions and needs a cleared buffer
-    if (use_rope &&
+    // only the in-tile RoPE kernel accumulates dQ with reductions and needs a cleared buffer
+    if (use_rope && !rotated_copies &&
         cudaMemsetAsync(dq_acc, 0, sizeof(float) * (size_t)T * Hq * D, stream) != cudaSuccess)
       return PK_ERR_CUDA;
   }
@@ -531,10 +532,24 @@ extern "C" int pk_attn_bwd(const void* dout, const void* q, const void* k, const
   if (!make_tile_map_bf16(&tq, q, T, Hq * D) || !make_tile_map_bf16(&tk, k, T, Hkv * D) ||
       !make_tile_map_bf16(&tv, v, T, Hkv * D) || !make_tile_map_bf16(&tdo, dout, T, Hq * D))
     return PK_ERR_CUDA;
+  if (rotated_copies) {
+    // rotated fp16 copies of q and k in the dQ accumulator section (not needed otherwise here)
+    char* qr = ws + lay.off[PK_WS_DQ_ACC];
+    char* kr = qr + align_up((size_t)T * Hq * D * 2, 256);
+    rc = rope_rotate_f16_launch(q, position_ids, T, Hq, D, rope_theta, qr, stream);
+    if (rc != PK_OK) return rc;
+    rc = rope_rotate_f16_launch(k, position_ids, T, Hkv, D, rope_theta, kr, stream);
+    if (rc != PK_OK) return rc;
+    CUtensorMap tqr, tkr;
+    if (!make_tile_map_bf16(&tqr, qr, T, Hq * D) || !make_tile_map_bf16(&tkr, kr, T, Hkv * D))
+      return PK_ERR_CUDA;
+    return launch_bwd_ws(tqr, tkr, tv, tdo, ws, lay, lse, dq, dk, dv, T, Hq, Hkv, D, grad_dtype,
+                         softmax_scale, true, stream);
+  }
   if (!use_rope) {
     // two warp-specialised kernels (dK/dV, then dQ); dQ is final, no finishing pass
     return launch_bwd_ws(tq, tk, tv, tdo, ws, lay, lse, dq, dk, dv, T, Hq, Hkv, D, grad_dtype,
-                         softmax_scale, stream);
+                         softmax_scale, false, stream);
   } else {
 #define PK_BWD(DD, RR, TT)                                                                      \
   rc = launch_bwd<DD, RR, TT>(tq, tk, tv, tdo, ws, lay, lse, dk, dv, T, Hq, Hkv, softmax_scale, \

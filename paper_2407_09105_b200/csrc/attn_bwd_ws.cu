@@ -79,13 +79,14 @@ enum DkvBar {
   kvSFull, kvDpFull, kvPReady, kvPReadyA, kvDsReady, kvUnitDone, kvDkvRead, kvNumBars
 };
 
-template <int D, typename GradT>
+template <int D, bool kRot, typename GradT>
 __global__ void __launch_bounds__(kWsThreads, 1)
 attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                     const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_do,
                     const int4* __restrict__ items, const int32_t* __restrict__ order, int32_t* hdr,
                     const float* __restrict__ lse, const float* __restrict__ delta,
                     GradT* __restrict__ dk, GradT* __restrict__ dv,
+                    const float2* __restrict__ rope_table,
                     int T, int Hq, int Hkv, float scale, float scale_log2) {
   using L = DkvSmem<D>;
   extern __shared__ __align__(1024) uint8_t smem[];
@@ -193,8 +194,13 @@ attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     // The whole warp walks the schedule (so that addresses and descriptors stay warp-uniform);
     // one elected lane issues the tensor-core instructions.
     {
-      constexpr uint32_t kIdescS = make_idesc(128, 128, kFmtBF16, kFmtBF16, 0, 0);
-      constexpr uint32_t kIdescKV = make_idesc(128, D, kFmtBF16, kFmtBF16, 0, 1);
+      // kRot: q and k are the rotated fp16 copies; dS then follows their format (operands of one
+      // contraction must share a format), everything touching V, dO and P stays bf16
+      constexpr uint32_t kQKFmt = kRot ? kFmtF16 : kFmtBF16;
+      constexpr uint32_t kIdescS = make_idesc(128, 128, kQKFmt, kQKFmt, 0, 0);
+      constexpr uint32_t kIdescDP = make_idesc(128, 128, kFmtBF16, kFmtBF16, 0, 0);
+      constexpr uint32_t kIdescDV = make_idesc(128, D, kFmtBF16, kFmtBF16, 0, 1);
+      constexpr uint32_t kIdescDK = make_idesc(128, D, kQKFmt, kQKFmt, 0, 1);
       const bool leader = elect_one();
       const uint32_t k_lo = desc_lo(sK, 16), v_lo = desc_lo(sV, 16), ds_lo = desc_lo(sdS, 16);
       int gs = 0, uc = 0;
@@ -216,7 +222,7 @@ attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 #pragma unroll
           for (int kk = 0; kk < D / 16; ++kk) {
             const uint32_t off = ((kk / 4) * L::kBoxBytes + (kk % 4) * 32) >> 4;
-            mma_ss(tdP, desc_from_lo(v_lo + off), desc_from_lo(do_lo + off), kIdescS, kk > 0);
+            mma_ss(tdP, desc_from_lo(v_lo + off), desc_from_lo(do_lo + off), kIdescDP, kk > 0);
           }
           mma_commit(bar(kvDpFull));
         }
@@ -249,7 +255,7 @@ attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           if (leader) {
 #pragma unroll
             for (int kk = 0; kk < kBM / 32; ++kk)   // dV += P^T dO, first half of the query rows
-              mma_ts(tdV, tS + kk * 8, desc_from_lo(doT_lo + ((kk * 2048) >> 4)), kIdescKV,
+              mma_ts(tdV, tS + kk * 8, desc_from_lo(doT_lo + ((kk * 2048) >> 4)), kIdescDV,
                      acc | (kk > 0));
           }
           __syncwarp();
@@ -258,7 +264,7 @@ attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           if (leader) {
 #pragma unroll
             for (int kk = kBM / 32; kk < kBM / 16; ++kk)
-              mma_ts(tdV, tS + kk * 8, desc_from_lo(doT_lo + ((kk * 2048) >> 4)), kIdescKV, 1u);
+              mma_ts(tdV, tS + kk * 8, desc_from_lo(doT_lo + ((kk * 2048) >> 4)), kIdescDV, 1u);
           }
           __syncwarp();
           const bool more = (s + 1 < n_steps);
@@ -275,7 +281,7 @@ attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             for (int kk = 0; kk < kBM / 16; ++kk) {   // dK += dS^T Q
               const uint32_t off = ((kk / 4) * L::kBoxBytes + (kk % 4) * 32) >> 4;
               mma_ss(tdK, desc_from_lo(ds_lo + off), desc_from_lo(qT_lo + ((kk * 2048) >> 4)),
-                     kIdescKV, acc | (kk > 0));
+                     kIdescDK, acc | (kk > 0));
             }
             mma_commit(bar(kvQdoEmpty0 + st));
           }
@@ -376,8 +382,8 @@ attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
               const float d1 = p[c2 * 32 + e + 1] * (__uint_as_float(dp[e + 1]) - d4.y);
               const float d2 = p[c2 * 32 + e + 2] * (__uint_as_float(dp[e + 2]) - d4.z);
               const float d3 = p[c2 * 32 + e + 3] * (__uint_as_float(dp[e + 3]) - d4.w);
-              dd[e >> 1] = pack_bf16x2(d0, d1);
-              dd[(e >> 1) + 1] = pack_bf16x2(d2, d3);
+              dd[e >> 1] = kRot ? pack_f16x2(d0, d1) : pack_bf16x2(d0, d1);
+              dd[(e >> 1) + 1] = kRot ? pack_f16x2(d2, d3) : pack_bf16x2(d2, d3);
             }
 #pragma unroll
             for (int ch = 0; ch < 4; ++ch) {
@@ -404,15 +410,40 @@ attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         GradT* dst = (is_dv ? dv : dk) + ((size_t)tok * Hkv + g) * D + col0;
         const uint32_t src = (is_dv ? tdV : tdK) + lane_off + col0;
         const float mul = is_dv ? 1.f : scale;
+        if (kRot && !is_dv) {
+          // dK was formed against the rotated k: rotate back by -angle, pairs (i, i + D/2)
+          static_assert(!kRot || (D == 128 && kEpiCols == 128), "rotated path is built for D = 128");
 #pragma unroll
-        for (int c = 0; c < kEpiCols / 32; ++c) {
-          uint32_t x[32];
-          float y[32];
-          tmem_ld32(src + c * 32, x);
-          tmem_wait_ld();
+          for (int c = 0; c < 2; ++c) {
+            uint32_t x1[32], x2[32];
+            float y1[32], y2[32];
+            tmem_ld32(src + c * 32, x1);
+            tmem_ld32(src + 64 + c * 32, x2);
+            tmem_wait_ld();
+            if (live) {
+              const float2* cs = rope_table + (size_t)tok * (D / 2) + c * 32;
 #pragma unroll
-          for (int e = 0; e < 32; ++e) y[e] = __uint_as_float(x[e]) * mul;
-          if (live) store_chunk32<GradT>(dst + c * 32, y);
+              for (int e = 0; e < 32; ++e) {
+                const float2 t = __ldg(cs + e);
+                const float a = __uint_as_float(x1[e]) * mul, b = __uint_as_float(x2[e]) * mul;
+                y1[e] = a * t.x + b * t.y;
+                y2[e] = b * t.x - a * t.y;
+              }
+              store_chunk32<GradT>(dst + c * 32, y1);
+              store_chunk32<GradT>(dst + 64 + c * 32, y2);
+            }
+          }
+        } else {
+#pragma unroll
+          for (int c = 0; c < kEpiCols / 32; ++c) {
+            uint32_t x[32];
+            float y[32];
+            tmem_ld32(src + c * 32, x);
+            tmem_wait_ld();
+#pragma unroll
+            for (int e = 0; e < 32; ++e) y[e] = __uint_as_float(x[e]) * mul;
+            if (live) store_chunk32<GradT>(dst + c * 32, y);
+          }
         }
       }
       tc_fence_before();
@@ -457,13 +488,14 @@ enum DqBar {
 // They are copied once per unit from shared memory into tensor memory, so that those two
 // contractions read only K / V from shared memory (the shared-memory port, not the tensor
 // pipe, was the bound when all four operands came from there).
-template <int D, typename GradT>
+template <int D, bool kRot, typename GradT>
 __global__ void __launch_bounds__(kWsThreads, 1)
 attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                    const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_do,
                    const int4* __restrict__ items, const int32_t* __restrict__ order, int32_t* hdr,
                    const float* __restrict__ lse, const float* __restrict__ delta,
-                   GradT* __restrict__ dq, int T, int Hq, int Hkv, float scale, float scale_log2) {
+                   GradT* __restrict__ dq, const float2* __restrict__ rope_table, int T, int Hq,
+                   int Hkv, float scale, float scale_log2) {
   using L = DqSmem<D>;
   extern __shared__ __align__(1024) uint8_t smem[];
   const uint32_t sbase = smem_u32(smem);
@@ -553,8 +585,10 @@ attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
     // The whole warp walks the schedule (so that addresses and descriptors stay warp-uniform);
     // one elected lane issues the tensor-core instructions.
     {
-      constexpr uint32_t kIdescS = make_idesc(128, 128, kFmtBF16, kFmtBF16, 0, 0);
-      constexpr uint32_t kIdescDQ = make_idesc(128, D, kFmtBF16, kFmtBF16, 0, 1);
+      constexpr uint32_t kQKFmt = kRot ? kFmtF16 : kFmtBF16;   // rotated q, k copies are fp16
+      constexpr uint32_t kIdescS = make_idesc(128, 128, kQKFmt, kQKFmt, 0, 0);
+      constexpr uint32_t kIdescDP = make_idesc(128, 128, kFmtBF16, kFmtBF16, 0, 0);
+      constexpr uint32_t kIdescDQ = make_idesc(128, D, kQKFmt, kQKFmt, 0, 1);   // dS follows k
       const bool leader = elect_one();
       int gk = 0, uc = 0;
       auto issue_s = [&](int g_idx) {       // S = Q K^T, Q from tensor memory
@@ -581,7 +615,7 @@ attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
 #pragma unroll
           for (int kk = 0; kk < D / 16; ++kk) {
             const uint32_t off = (kk / 4) * L::kBoxBytes + (kk % 4) * 32;
-            mma_ts(tdP, tdO + kk * 8, desc_from_lo(v_lo + (off >> 4)), kIdescS, kk > 0);
+            mma_ts(tdP, tdO + kk * 8, desc_from_lo(v_lo + (off >> 4)), kIdescDP, kk > 0);
           }
           mma_commit(bar(dqDpFull));
           mma_commit(bar(dqVEmpty0 + vs));
@@ -696,7 +730,7 @@ attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
           for (int e = 0; e < 32; e += 2) {
             const float d0 = p[c2 * 32 + e] * (__uint_as_float(dp[e]) - dl);
             const float d1 = p[c2 * 32 + e + 1] * (__uint_as_float(dp[e + 1]) - dl);
-            dd[c2 * 16 + (e >> 1)] = pack_bf16x2(d0, d1);
+            dd[c2 * 16 + (e >> 1)] = kRot ? pack_f16x2(d0, d1) : pack_bf16x2(d0, d1);
           }
         }
         // every thread must have read dP before dS overwrites its columns
@@ -714,16 +748,39 @@ attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
       tc_fence_after();
       if (qd < 2) {
         const bool live = (row < q_len) && (*s_abort == 0);
-        GradT* dst = dq + ((size_t)tok * Hq + h) * D + qd * (D / 2);
-#pragma unroll
-        for (int c = 0; c < D / 64; ++c) {
-          uint32_t x[32];
-          float y[32];
-          tmem_ld32(tdQ + lane_off + qd * (D / 2) + c * 32, x);
+        if (kRot) {
+          // rotate back by -angle: this thread owns pairs i in [32*qd, +32) and i + 64
+          static_assert(!kRot || D == 128, "rotated path is built for D = 128");
+          GradT* dst = dq + ((size_t)tok * Hq + h) * D + qd * 32;
+          uint32_t x1[32], x2[32];
+          float y1[32], y2[32];
+          tmem_ld32(tdQ + lane_off + qd * 32, x1);
+          tmem_ld32(tdQ + lane_off + 64 + qd * 32, x2);
           tmem_wait_ld();
+          if (live) {
+            const float2* cs = rope_table + (size_t)tok * (D / 2) + qd * 32;
 #pragma unroll
-          for (int e = 0; e < 32; ++e) y[e] = __uint_as_float(x[e]) * scale;
-          if (live) store_chunk32<GradT>(dst + c * 32, y);
+            for (int e = 0; e < 32; ++e) {
+              const float2 t = __ldg(cs + e);
+              const float a = __uint_as_float(x1[e]) * scale, b = __uint_as_float(x2[e]) * scale;
+              y1[e] = a * t.x + b * t.y;
+              y2[e] = b * t.x - a * t.y;
+            }
+            store_chunk32<GradT>(dst, y1);
+            store_chunk32<GradT>(dst + 64, y2);
+          }
+        } else {
+          GradT* dst = dq + ((size_t)tok * Hq + h) * D + qd * (D / 2);
+#pragma unroll
+          for (int c = 0; c < D / 64; ++c) {
+            uint32_t x[32];
+            float y[32];
+            tmem_ld32(tdQ + lane_off + qd * (D / 2) + c * 32, x);
+            tmem_wait_ld();
+#pragma unroll
+            for (int e = 0; e < 32; ++e) y[e] = __uint_as_float(x[e]) * scale;
+            if (live) store_chunk32<GradT>(dst + c * 32, y);
+          }
         }
       }
       tc_fence_before();
@@ -737,13 +794,13 @@ attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
   if (warp == kMmaWarp) tmem_dealloc(tmem, 512);
 }
 
-template <int D, typename GradT>
+template <int D, bool kRot, typename GradT>
 int launch_ws(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
               const CUtensorMap& tdo, char* ws, const WorkspaceLayout& lay, const float* lse,
               void* dq, void* dk, void* dv, int T, int Hq, int Hkv, float scale,
               cudaStream_t stream) {
-  auto kern_kv = attn_bwd_dkv_kernel<D, GradT>;
-  auto kern_q = attn_bwd_dq_kernel<D, GradT>;
+  auto kern_kv = attn_bwd_dkv_kernel<D, kRot, GradT>;
+  auto kern_q = attn_bwd_dq_kernel<D, kRot, GradT>;
   if (cudaFuncSetAttribute(kern_kv, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            DkvSmem<D>::kTotal) != cudaSuccess ||
       cudaFuncSetAttribute(kern_q, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -751,13 +808,15 @@ int launch_ws(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& t
     return PK_ERR_CUDA;
   int32_t* hdr = reinterpret_cast<int32_t*>(ws + lay.off[PK_WS_HEADER]);
   const float* delta = reinterpret_cast<const float*>(ws + lay.off[PK_WS_DELTA]);
+  const float2* table = reinterpret_cast<const float2*>(ws + lay.off[PK_WS_ROPE_TABLE]);
   const int grid = sm_count();
   {
     TimedLaunch timed(PK_KERNEL_BWD, stream);
     kern_kv<<<grid, kWsThreads, DkvSmem<D>::kTotal, stream>>>(
         tq, tk, tv, tdo, reinterpret_cast<const int4*>(ws + lay.off[PK_WS_BWD_ITEMS]),
         reinterpret_cast<const int32_t*>(ws + lay.off[PK_WS_BWD_ORDER]), hdr, lse, delta,
-        static_cast<GradT*>(dk), static_cast<GradT*>(dv), T, Hq, Hkv, scale, scale * kLog2eWs);
+        static_cast<GradT*>(dk), static_cast<GradT*>(dv), table, T, Hq, Hkv, scale,
+        scale * kLog2eWs);
   }
   if (launch_status() != PK_OK) return PK_ERR_CUDA;
   {
@@ -765,7 +824,7 @@ int launch_ws(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& t
     kern_q<<<grid, kWsThreads, DqSmem<D>::kTotal, stream>>>(
         tq, tk, tv, tdo, reinterpret_cast<const int4*>(ws + lay.off[PK_WS_FWD_ITEMS]),
         reinterpret_cast<const int32_t*>(ws + lay.off[PK_WS_FWD_ORDER]), hdr, lse, delta,
-        static_cast<GradT*>(dq), T, Hq, Hkv, scale, scale * kLog2eWs);
+        static_cast<GradT*>(dq), table, T, Hq, Hkv, scale, scale * kLog2eWs);
   }
   return launch_status();
 }
@@ -775,18 +834,20 @@ int launch_ws(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& t
 int launch_bwd_ws(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
                   const CUtensorMap& tdo, char* ws, const WorkspaceLayout& lay, const float* lse,
                   void* dq, void* dk, void* dv, int T, int Hq, int Hkv, int D, int grad_dtype,
-                  float scale, cudaStream_t stream) {
+                  float scale, bool rotated, cudaStream_t stream) {
+#define PK_BWS(DD, RR, TT)                                                                     \
+  return launch_ws<DD, RR, TT>(tq, tk, tv, tdo, ws, lay, lse, dq, dk, dv, T, Hq, Hkv, scale, \
+                               stream)
   if (D == 128) {
-    if (grad_dtype == PK_BF16)
-      return launch_ws<128, __nv_bfloat16>(tq, tk, tv, tdo, ws, lay, lse, dq, dk, dv, T, Hq, Hkv,
-                                           scale, stream);
-    return launch_ws<128, float>(tq, tk, tv, tdo, ws, lay, lse, dq, dk, dv, T, Hq, Hkv, scale,
-                                 stream);
+    if (rotated) {
+      if (grad_dtype == PK_BF16) PK_BWS(128, true, __nv_bfloat16); else PK_BWS(128, true, float);
+    } else {
+      if (grad_dtype == PK_BF16) PK_BWS(128, false, __nv_bfloat16); else PK_BWS(128, false, float);
+    }
   }
-  if (grad_dtype == PK_BF16)
-    return launch_ws<64, __nv_bfloat16>(tq, tk, tv, tdo, ws, lay, lse, dq, dk, dv, T, Hq, Hkv,
-                                        scale, stream);
-  return launch_ws<64, float>(tq, tk, tv, tdo, ws, lay, lse, dq, dk, dv, T, Hq, Hkv, scale, stream);
+  if (grad_dtype == PK_BF16) PK_BWS(64, false, __nv_bfloat16);
+  PK_BWS(64, false, float);
+#undef PK_BWS
 }
 
 }  // namespace pk

@@ -357,6 +357,22 @@ extern "C" int pk_attn_fwd(const void* q, const void* k, const void* v,
     if (rc != PK_OK) return rc;
   }
   const bool use_rope = rope_theta > 0.f;
+  const bool ws_shape = (Hq / Hkv) % 2 == 0;
+  if (use_rope && g_rope_mode == PK_ROPE_ROTATED_COPIES && D == 128 && ws_shape) {
+    // rotated fp16 copies of q and k in the (otherwise unused) dQ accumulator section
+    char* qr = ws + lay.off[PK_WS_DQ_ACC];
+    char* kr = qr + align_up((size_t)T * Hq * D * 2, 256);
+    int rc = rope_rotate_f16_launch(q, position_ids, T, Hq, D, rope_theta, qr, stream);
+    if (rc != PK_OK) return rc;
+    rc = rope_rotate_f16_launch(k, position_ids, T, Hkv, D, rope_theta, kr, stream);
+    if (rc != PK_OK) return rc;
+    CUtensorMap tqr, tkr, tvv;
+    if (!make_tile_map_bf16(&tqr, qr, T, Hq * D) || !make_tile_map_bf16(&tkr, kr, T, Hkv * D) ||
+        !make_tile_map_bf16(&tvv, v, T, Hkv * D))
+      return PK_ERR_CUDA;
+    return launch_fwd_ws(tqr, tkr, tvv, ws, lay, out, lse, T, Hq, Hkv, D, out_dtype, softmax_scale,
+                         true, stream);
+  }
   if (use_rope) {
     int rc = rope_table_launch(position_ids, T, D, rope_theta,
                                reinterpret_cast<float*>(ws + lay.off[PK_WS_ROPE_TABLE]), stream);
@@ -367,9 +383,9 @@ extern "C" int pk_attn_fwd(const void* q, const void* k, const void* v,
       !make_tile_map_bf16(&tv, v, T, Hkv * D))
     return PK_ERR_CUDA;
 
-  if (!use_rope && (Hq / Hkv) % 2 == 0)   // two query heads of a kv head per CTA, warp-specialised
+  if (!use_rope && ws_shape)   // two query heads of a kv head per CTA, warp-specialised
     return launch_fwd_ws(tq, tk, tv, ws, lay, out, lse, T, Hq, Hkv, D, out_dtype, softmax_scale,
-                         stream);
+                         false, stream);
 #define PK_FWD(DD, RR, TT) \
   return launch_fwd<DD, RR, TT>(tq, tk, tv, ws, lay, out, lse, T, Hq, Hkv, softmax_scale, stream)
   if (D == 128) {

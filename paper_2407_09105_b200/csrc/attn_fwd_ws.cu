@@ -61,7 +61,7 @@ __device__ __forceinline__ void store_out32(OutT* dst, const uint32_t* r, float 
   store_chunk32<OutT>(dst, y);
 }
 
-template <int D, typename OutT>
+template <int D, bool kRot, typename OutT>
 __global__ void __launch_bounds__(kFwsThreads, 1)
 attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                    const __grid_constant__ CUtensorMap tm_v, const int4* __restrict__ items,
@@ -154,7 +154,9 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
     // The whole warp walks the schedule (so that addresses and descriptors stay warp-uniform);
     // one elected lane issues the tensor-core instructions.
     {
-      constexpr uint32_t kIdescQK = make_idesc(128, 128, kFmtBF16, kFmtBF16, 0, 0);
+      // kRot: q and k are the rotated fp16 copies in the workspace
+      constexpr uint32_t kQKFmt = kRot ? kFmtF16 : kFmtBF16;
+      constexpr uint32_t kIdescQK = make_idesc(128, 128, kQKFmt, kQKFmt, 0, 0);
       constexpr uint32_t kIdescPV = make_idesc(128, D, kFmtBF16, kFmtBF16, 0, 1);
       const bool leader = elect_one();
       int gk = 0, uc = 0;
@@ -315,11 +317,11 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
   if (warp == kFwsMmaWarp) tmem_dealloc(tmem, 512);
 }
 
-template <int D, typename OutT>
+template <int D, bool kRot, typename OutT>
 int launch_fws(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, char* ws,
                const WorkspaceLayout& lay, void* out, float* lse, int T, int Hq, int Hkv,
                float scale, cudaStream_t stream) {
-  auto kern = attn_fwd_ws_kernel<D, OutT>;
+  auto kern = attn_fwd_ws_kernel<D, kRot, OutT>;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            FwsSmem<D>::kTotal) != cudaSuccess)
     return PK_ERR_CUDA;
@@ -336,15 +338,19 @@ int launch_fws(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& 
 
 int launch_fwd_ws(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, char* ws,
                   const WorkspaceLayout& lay, void* out, float* lse, int T, int Hq, int Hkv, int D,
-                  int out_dtype, float scale, cudaStream_t stream) {
+                  int out_dtype, float scale, bool rotated, cudaStream_t stream) {
+#define PK_FWS(DD, RR, TT) \
+  return launch_fws<DD, RR, TT>(tq, tk, tv, ws, lay, out, lse, T, Hq, Hkv, scale, stream)
   if (D == 128) {
-    if (out_dtype == PK_BF16)
-      return launch_fws<128, __nv_bfloat16>(tq, tk, tv, ws, lay, out, lse, T, Hq, Hkv, scale, stream);
-    return launch_fws<128, float>(tq, tk, tv, ws, lay, out, lse, T, Hq, Hkv, scale, stream);
+    if (rotated) {
+      if (out_dtype == PK_BF16) PK_FWS(128, true, __nv_bfloat16); else PK_FWS(128, true, float);
+    } else {
+      if (out_dtype == PK_BF16) PK_FWS(128, false, __nv_bfloat16); else PK_FWS(128, false, float);
+    }
   }
-  if (out_dtype == PK_BF16)
-    return launch_fws<64, __nv_bfloat16>(tq, tk, tv, ws, lay, out, lse, T, Hq, Hkv, scale, stream);
-  return launch_fws<64, float>(tq, tk, tv, ws, lay, out, lse, T, Hq, Hkv, scale, stream);
+  if (out_dtype == PK_BF16) PK_FWS(64, false, __nv_bfloat16);
+  PK_FWS(64, false, float);
+#undef PK_FWS
 }
 
 }  // namespace pk

@@ -4,6 +4,7 @@
 // Sec. 3.5); the rotation is the usual half-split one.  Angles are formed in fp64 so
 // that ids up to 2^17 lose nothing before the fp32 cos/sin are taken.
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 
 #include "pk_common.cuh"
 
@@ -50,7 +51,41 @@ __global__ void rope_apply_kernel(__nv_bfloat16* __restrict__ x, const int32_t* 
   }
 }
 
+// y = rotate(x) stored as fp16: one thread per (token, pair index), looping over the heads.
+__global__ void rope_rotate_f16_kernel(const __nv_bfloat16* __restrict__ x,
+                                       const int32_t* __restrict__ pos, int T, int H, int D,
+                                       double log2_theta, __half* __restrict__ y) {
+  const int half = D / 2;
+  const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= (int64_t)T * half) return;
+  const int t = (int)(idx / half), i = (int)(idx % half);
+  float c, s;
+  angle_cos_sin(pos[t], i, D, log2_theta, &c, &s);
+  const __nv_bfloat16* xr = x + (int64_t)t * H * D;
+  __half* yr = y + (int64_t)t * H * D;
+  for (int h = 0; h < H; ++h) {
+    const float a = __bfloat162float(xr[h * D + i]);
+    const float b = __bfloat162float(xr[h * D + i + half]);
+    yr[h * D + i] = __float2half_rn(a * c - b * s);
+    yr[h * D + i + half] = __float2half_rn(b * c + a * s);
+  }
+}
+
 }  // namespace
+
+int g_rope_mode = 0;
+
+int rope_rotate_f16_launch(const void* x, const int32_t* position_ids, int32_t T, int32_t H,
+                           int32_t D, float theta, void* y, cudaStream_t stream) {
+  if (T == 0) return PK_OK;
+  const int64_t n = (int64_t)T * (D / 2);
+  const int threads = 256;
+  const unsigned blocks = (unsigned)((n + threads - 1) / threads);
+  rope_rotate_f16_kernel<<<blocks, threads, 0, stream>>>(
+      static_cast<const __nv_bfloat16*>(x), position_ids, T, H, D, log2((double)theta),
+      static_cast<__half*>(y));
+  return launch_status();
+}
 
 int rope_table_launch(const int32_t* position_ids, int32_t T, int32_t D, float theta,
                       float* table, cudaStream_t stream) {
@@ -78,4 +113,10 @@ extern "C" int pk_rope_apply(void* x, const int32_t* position_ids, int32_t T, in
   pk::rope_apply_kernel<<<blocks, threads, 0, static_cast<cudaStream_t>(stream)>>>(
       static_cast<__nv_bfloat16*>(x), position_ids, T, H, D, log2((double)theta), inverse);
   return pk::launch_status();
+}
+
+extern "C" int pk_set_rope_mode(int32_t mode) {
+  if (mode != PK_ROPE_ROTATED_COPIES && mode != PK_ROPE_IN_TILE) return PK_ERR_INVALID_ARG;
+  pk::g_rope_mode = mode;
+  return PK_OK;
 }

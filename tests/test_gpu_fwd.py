@@ -48,9 +48,15 @@ def test_gqa(D):
     _case([200, 77, 400], 8, 2, D, 0.0, seed=4)
 
 
+@pytest.mark.parametrize("mode", [api.PK_ROPE_ROTATED_COPIES, api.PK_ROPE_IN_TILE])
 @pytest.mark.parametrize("D,theta", [(64, 1e4), (128, 1e4), (128, 5e5)])
-def test_fused_rope(D, theta):
-    _case([150, 260, 3, 129], 4, 2, D, theta, seed=5)
+def test_fused_rope(D, theta, mode):
+    api.pk_set_rope_mode(mode)
+    try:
+        _case([150, 260, 3, 129], 4, 2, D, theta, seed=5)
+        _case([300, 40], 4, 4, D, theta, seed=15)          # MHA: the forward stays in-tile
+    finally:
+        api.pk_set_rope_mode(api.PK_ROPE_ROTATED_COPIES)
 
 
 def test_rope_uses_given_ids_of_a_fragment():
