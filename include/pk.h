@@ -52,7 +52,7 @@ extern "C" {
 #define PK_WS_HEADER     0   /* int32[32]: see PK_HDR_* indices                        */
 #define PK_WS_FWD_ITEMS  1   /* int32[T][4]  (q_start, q_len, kv_start, kv_len)        */
 #define PK_WS_BWD_ITEMS  2   /* int32[T][4]  (kv_start, kv_len, q_start, q_len)        */
-#define PK_WS_FWD_ORDER  3   /* int32[T]     item indices, longest work first          */
+#define PK_WS_FWD_ORDER  3   /* int32[T]     item indices, longest example first       */
 #define PK_WS_BWD_ORDER  4   /* int32[T]                                                */
 #define PK_WS_DELTA      5   /* fp32 [Hq][T] row sums of dO*O                           */
 #define PK_WS_DQ_ACC     6   /* fp32 [T+128][Hq][D] accumulator of dQ                   */
@@ -99,8 +99,9 @@ int pk_workspace_section(int32_t which, int32_t T, int32_t Hq, int32_t Hkv, int3
  *                 plan: forward items (a block of <= bm query rows of one example and
  *                 the key range [example start, last row] it may see), backward items
  *                 (a block of <= bn key rows and the query range up to the example end
- *                 that may see it), both in ascending (example, block) order, plus for
- *                 each list the stable permutation by descending number of tiles.
+ *                 that may see it), both in ascending (example, block) order, plus the
+ *                 schedule order of the items: stable sort by descending tile count of the
+ *                 item's example (long examples first, an example's items adjacent).
  * T == 0 is valid: cu_seqlens = [0], E = 0.  No host round trip; one kernel launch.
  */
 int pk_seqlens_from_posids(const int32_t* position_ids, int32_t T,

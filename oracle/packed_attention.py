@@ -74,9 +74,11 @@ def work_lists(cu_seqlens, n_examples, bm, bn):
         rows of one example together with the key range it may see.
     backward item (kv_start, kv_len, q_start, q_len): a block of <= bn key rows
         of one example together with the query range that may see it.
-    ``*_order`` is the stable sort of the item indices by descending number of
-    tiles the item visits (longest work first).
+    ``*_order`` is the stable sort of the item indices by descending tile count of the
+    item's EXAMPLE (ceil(L_e / bm)): long examples first, the items of one example adjacent
+    and in block order.  Both lists have the same order.
     """
+    assert bm == bn, "the lists are defined for square tiles"
     fwd, bwd = [], []
     for e in range(n_examples):
         s, t = int(cu_seqlens[e]), int(cu_seqlens[e + 1])
@@ -93,10 +95,13 @@ def work_lists(cu_seqlens, n_examples, bm, bn):
             b += 1
     fwd = np.asarray(fwd, dtype=np.int32).reshape(-1, 4)
     bwd = np.asarray(bwd, dtype=np.int32).reshape(-1, 4)
-    fwd_tiles = [-(-int(it[3]) // bn) for it in fwd]
-    bwd_tiles = [-(-int(it[3]) // bm) for it in bwd]
-    fwd_order = np.asarray(sorted(range(len(fwd)), key=lambda i: -fwd_tiles[i]), dtype=np.int32)
-    bwd_order = np.asarray(sorted(range(len(bwd)), key=lambda i: -bwd_tiles[i]), dtype=np.int32)
+    ex_tiles = []
+    for e in range(n_examples):
+        n = -(-(int(cu_seqlens[e + 1]) - int(cu_seqlens[e])) // bm)
+        ex_tiles.extend([n] * n)
+    order = sorted(range(len(fwd)), key=lambda i: -ex_tiles[i])      # sorted() is stable
+    fwd_order = np.asarray(order, dtype=np.int32)
+    bwd_order = np.asarray(order, dtype=np.int32)
     return fwd, bwd, fwd_order, bwd_order
 
 

@@ -115,8 +115,9 @@ plan_kernel(const int32_t* __restrict__ pos, int T,
     const int blk_len = min(kBM, L - b * kBM);
     fwd_items[n] = make_int4(s + b * kBM, blk_len, s, b * kBM + blk_len);
     bwd_items[n] = make_int4(s + b * kBN, blk_len, s + b * kBN, L - b * kBN);
-    atomicAdd(&hist_f[b + 1], 1);
-    atomicAdd(&hist_b[(L - b * kBN + kBM - 1) / kBM], 1);
+    // sort key of both lists: the tile count of the item's EXAMPLE (see phase E)
+    atomicAdd(&hist_f[(L + kBM - 1) / kBM], 1);
+    atomicAdd(&hist_b[(L + kBM - 1) / kBM], 1);
   }
   __syncthreads();
 
@@ -137,12 +138,19 @@ plan_kernel(const int32_t* __restrict__ pos, int T,
   __syncthreads();
 
   // ---- E: stable placement: chunks in order, warps of a chunk in order --------------
+  // Items are ordered by descending tile count of their example and, inside an example, by
+  // block: long examples first (their items carry the most work) while the units that run at
+  // the same time belong to the same example and share its K/V (or Q/dO) tiles in L2.
   for (int base = 0; base < N; base += kPlanThreads) {
     const int n = base + tid;
     int kf = 0, kb = 0;
     if (n < N) {
-      kf = (fwd_items[n].w + kBN - 1) / kBN;
-      kb = (bwd_items[n].w + kBM - 1) / kBM;
+      int lo = 0, hi = E - 1;
+      while (lo < hi) {
+        const int mid = (lo + hi + 1) >> 1;
+        if (ex_base[mid] <= n) lo = mid; else hi = mid - 1;
+      }
+      kf = kb = ex_base[lo + 1] - ex_base[lo];
     }
     for (int w = 0; w < kPlanThreads / 32; ++w) {
       if (warp == w) {

@@ -120,14 +120,16 @@ def test_work_lists_cover_exactly_the_mask(bm, bn, lens):
     # closed forms for the counts
     assert len(fwd) == sum(-(-l // bm) for l in lens)
     assert len(bwd) == sum(-(-l // bn) for l in lens)
-    # order: permutation, non-increasing tile counts, ties in index order
-    ft = [-(-int(x[3]) // bn) for x in fwd]
-    assert sorted(fo.tolist()) == list(range(len(fwd)))
-    keys = [(-ft[i], i) for i in fo]
+    # order: a permutation; examples by descending tile count (ties in stream order), the items
+    # of an example adjacent and in block order
+    ex_of = [int(eid[x[0]]) for x in fwd]
+    ex_tiles = [sum(1 for y in ex_of if y == e) for e in ex_of]
+    assert sorted(fo.tolist()) == list(range(len(fwd))) and fo.tolist() == bo.tolist()
+    keys = [(-ex_tiles[i], i) for i in fo]
     assert keys == sorted(keys)
-    bt = [-(-int(x[3]) // bm) for x in bwd]
-    keys = [(-bt[i], i) for i in bo]
-    assert keys == sorted(keys) and sorted(bo.tolist()) == list(range(len(bwd)))
+    for a, b in zip(fo[:-1], fo[1:]):
+        if ex_of[a] == ex_of[b]:
+            assert b == a + 1
 
 
 def test_work_list_visit_counts_match_closed_form():
