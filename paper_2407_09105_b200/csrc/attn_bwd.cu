@@ -30,32 +30,45 @@ constexpr int kBwdThreads = 128;
 constexpr float kLog2e = 1.4426950408889634f;
 
 // ------------------------------------------------------------------ delta pre-pass
-// One warp per (token, head) row; lanes split the row, shuffles reduce it.
+// D/8 lanes per (token, head) row, 16 bytes of dO per lane; shuffles reduce inside the lane
+// group (a warp covers 32*8/D rows).  HBM-bound: reads dO and O once.
 template <typename OutT>
 __global__ void delta_kernel(const __nv_bfloat16* __restrict__ dout, const OutT* __restrict__ out,
                              float* __restrict__ delta, int T, int Hq, int D) {
-  const int64_t row = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const int lanes_per_row = D >> 3;                       // 16 (D = 128) or 8 (D = 64)
+  const int rows_per_warp = 32 / lanes_per_row;
   const int lane = threadIdx.x & 31;
-  if (row >= (int64_t)T * Hq) return;
-  const __nv_bfloat16* a = dout + row * D;
-  const OutT* b = out + row * D;
+  const int64_t warp_id = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const int64_t row = warp_id * rows_per_warp + lane / lanes_per_row;
+  const int c = (lane % lanes_per_row) * 8;
   float acc = 0.f;
-  for (int c = lane * 2; c < D; c += 64) {
-    const float2 x = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(a + c));
-    float y0, y1;
+  if (row < (int64_t)T * Hq) {
+    const uint4 a4 = *reinterpret_cast<const uint4*>(dout + row * D + c);
+    const __nv_bfloat162* av = reinterpret_cast<const __nv_bfloat162*>(&a4);
+    float y[8];
     if (sizeof(OutT) == 2) {
-      const float2 y = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(b + c));
-      y0 = y.x; y1 = y.y;
-    } else {
-      const float2 y = *reinterpret_cast<const float2*>(b + c);
-      y0 = y.x; y1 = y.y;
-    }
-    acc = fmaf(x.x, y0, acc);
-    acc = fmaf(x.y, y1, acc);
-  }
+      const uint4 b4 = *reinterpret_cast<const uint4*>(out + row * D + c);
+      const __nv_bfloat162* bv = reinterpret_cast<const __nv_bfloat162*>(&b4);
 #pragma unroll
-  for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-  if (lane == 0) {
+      for (int e = 0; e < 4; ++e) {
+        const float2 f = __bfloat1622float2(bv[e]);
+        y[2 * e] = f.x; y[2 * e + 1] = f.y;
+      }
+    } else {
+      const float4 b0 = *reinterpret_cast<const float4*>(out + row * D + c);
+      const float4 b1 = *reinterpret_cast<const float4*>(out + row * D + c + 4);
+      y[0] = b0.x; y[1] = b0.y; y[2] = b0.z; y[3] = b0.w;
+      y[4] = b1.x; y[5] = b1.y; y[6] = b1.z; y[7] = b1.w;
+    }
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const float2 x = __bfloat1622float2(av[e]);
+      acc = fmaf(x.x, y[2 * e], acc);
+      acc = fmaf(x.y, y[2 * e + 1], acc);
+    }
+  }
+  for (int o = lanes_per_row >> 1; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+  if ((lane % lanes_per_row) == 0 && row < (int64_t)T * Hq) {
     const int t = (int)(row / Hq), h = (int)(row % Hq);
     delta[(size_t)h * T + t] = acc;
   }
@@ -511,7 +524,8 @@ extern "C" int pk_attn_bwd(const void* dout, const void* q, const void* k, const
   {
     const int64_t rows = (int64_t)T * Hq;
     const int warps = 8;
-    const unsigned blocks = (unsigned)((rows + warps - 1) / warps);
+    const int64_t rows_per_block = (int64_t)warps * (32 / (D >> 3));
+    const unsigned blocks = (unsigned)((rows + rows_per_block - 1) / rows_per_block);
     TimedLaunch timed(PK_KERNEL_DELTA, stream);
     if (out_dtype == PK_BF16)
       delta_kernel<__nv_bfloat16><<<blocks, warps * 32, 0, stream>>>(

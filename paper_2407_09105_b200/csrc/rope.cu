@@ -56,6 +56,40 @@ __global__ void rope_rotate_f16_kernel(const __nv_bfloat16* __restrict__ x,
                                        const int32_t* __restrict__ pos, int T, int H, int D,
                                        double log2_theta, __half* __restrict__ y) {
   const int half = D / 2;
+  if ((D & 15) == 0) {
+    // 16-byte accesses: a thread owns 8 consecutive pair indices of one token; its 8 (cos, sin)
+    // are formed once and reused for every head.  HBM-bound: 2 B read + 2 B written per element.
+    const int chunks = half / 8;
+    const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= (int64_t)T * chunks) return;
+    const int t = (int)(idx / chunks), i0 = (int)(idx % chunks) * 8;
+    float c[8], s[8];
+    const int p = pos[t];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) angle_cos_sin(p, i0 + e, D, log2_theta, &c[e], &s[e]);
+    const __nv_bfloat16* xr = x + (int64_t)t * H * D + i0;
+    __half* yr = y + (int64_t)t * H * D + i0;
+    for (int h = 0; h < H; ++h) {
+      const uint4 a4 = *reinterpret_cast<const uint4*>(xr + h * D);
+      const uint4 b4 = *reinterpret_cast<const uint4*>(xr + h * D + half);
+      const __nv_bfloat162* av = reinterpret_cast<const __nv_bfloat162*>(&a4);
+      const __nv_bfloat162* bv = reinterpret_cast<const __nv_bfloat162*>(&b4);
+      uint4 o1, o2;
+      __half2* o1v = reinterpret_cast<__half2*>(&o1);
+      __half2* o2v = reinterpret_cast<__half2*>(&o2);
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const float2 a = __bfloat1622float2(av[e]), b = __bfloat1622float2(bv[e]);
+        o1v[e] = __floats2half2_rn(a.x * c[2 * e] - b.x * s[2 * e],
+                                   a.y * c[2 * e + 1] - b.y * s[2 * e + 1]);
+        o2v[e] = __floats2half2_rn(b.x * c[2 * e] + a.x * s[2 * e],
+                                   b.y * c[2 * e + 1] + a.y * s[2 * e + 1]);
+      }
+      *reinterpret_cast<uint4*>(yr + h * D) = o1;
+      *reinterpret_cast<uint4*>(yr + h * D + half) = o2;
+    }
+    return;
+  }
   const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (idx >= (int64_t)T * half) return;
   const int t = (int)(idx / half), i = (int)(idx % half);
@@ -78,8 +112,8 @@ int g_rope_mode = 0;
 int rope_rotate_f16_launch(const void* x, const int32_t* position_ids, int32_t T, int32_t H,
                            int32_t D, float theta, void* y, cudaStream_t stream) {
   if (T == 0) return PK_OK;
-  const int64_t n = (int64_t)T * (D / 2);
-  const int threads = 256;
+  const int64_t n = (int64_t)T * ((D & 15) == 0 ? D / 16 : D / 2);
+  const int threads = 128;
   const unsigned blocks = (unsigned)((n + threads - 1) / threads);
   rope_rotate_f16_kernel<<<blocks, threads, 0, stream>>>(
       static_cast<const __nv_bfloat16*>(x), position_ids, T, H, D, log2((double)theta),
