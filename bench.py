@@ -298,7 +298,9 @@ def main():
     ms_step = replicas.max_over_ranks(e0.elapsed_time(e1), dist, "cuda") / args.steps
     fwd_ms = float(np.mean([a.elapsed_time(b) for a, b in kev[api.PK_KERNEL_FWD]]))
     bwd_ms = float(np.mean([a.elapsed_time(b) for a, b in kev[api.PK_KERNEL_BWD]]))
-    dq_ms = float(np.mean([a.elapsed_time(b) for a, b in kev[api.PK_KERNEL_BWD_DQ]])) if theta <= 0 else 0.0
+    # two backward kernels unless the in-tile RoPE kernels run (RoPE with head_dim != 128)
+    split = theta <= 0 or D == 128
+    dq_ms = float(np.mean([a.elapsed_time(b) for a, b in kev[api.PK_KERNEL_BWD_DQ]])) if split else 0.0
 
     flops_step = w.useful_flops_fwd + w.useful_flops_bwd
     value = world * flops_step / (ms_step * 1e-3) / 1e12
@@ -345,7 +347,6 @@ def main():
     # without fused RoPE the backward is two kernels: dK/dV (6 of the 10 useful FLOPs per pair and
     # head-dim: dV, dK, plus one of the two recomputed products) and dQ.  The dominant kernel is
     # the dK/dV one; its useful work is dV and dK only: 4*D FLOPs per pair.
-    split = theta <= 0
     bwd_flops = (w.useful_flops_bwd * 4 // 10) if split else w.useful_flops_bwd
     bwd_tflops = bwd_flops / (bwd_ms * 1e-3) / 1e12
     executed = ((8 if split else 10) * D * Hq * w.causal_pairs) / (bwd_ms * 1e-3) / 1e12

@@ -662,20 +662,10 @@ attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
     const int row = tid & 127;              // query row inside the tile
     const int qd = tid >> 7;                // which group of kCW key columns
     const uint32_t lane_off = static_cast<uint32_t>((warp & 3) * 32) << 16;
-    int gk = 0, uc = 0;
-    for (int r = 0;; ++r, ++uc) {
-      const int u = snake_unit(r, cta, n_cta);
-      if (u >= n_units || *s_abort) break;
-      const int4 it = items[order[u / Hq]];
-      const int h = u % Hq;
-      const int q_start = it.x, q_len = it.y, kv_len = it.w;
-      const int n_kv = (kv_len + kBN - 1) / kBN;
-      const int tok = q_start + row;
-      const float lse2 = (tok < T) ? lse[(size_t)h * T + tok] * kLog2eWs : 0.f;
-      const float dl = (tok < T) ? delta[(size_t)h * T + tok] : 0.f;
-
-      // ---- Q and dO rows: shared memory (128B-swizzled) -> tensor memory, half a row per thread
-      mbar_wait(bar(dqQFull), uc & 1, s_abort);
+    // Q and dO rows of unit number `n`: shared memory (128B-swizzled) -> tensor memory, half a
+    // row per thread; then the shared-memory copies may be overwritten by the next load.
+    auto copy_q_do = [&](int n) {
+      mbar_wait(bar(dqQFull), n & 1, s_abort);
       if (qd < 2) {
         constexpr int kElems = D / 2;                       // elements per thread
         const int box = (qd * kElems) / 64, chunk0 = ((qd * kElems) % 64) / 8;
@@ -696,7 +686,20 @@ attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
       }
       tc_fence_before();
       mbar_arrive(bar(dqQtReady));
-      mbar_arrive(bar(dqQEmpty));      // the shared-memory copies may be overwritten
+      mbar_arrive(bar(dqQEmpty));
+    };
+    int gk = 0, uc = 0;
+    if (snake_unit(0, cta, n_cta) < n_units && !*s_abort) copy_q_do(0);
+    for (int r = 0;; ++r, ++uc) {
+      const int u = snake_unit(r, cta, n_cta);
+      if (u >= n_units || *s_abort) break;
+      const int4 it = items[order[u / Hq]];
+      const int h = u % Hq;
+      const int q_start = it.x, q_len = it.y, kv_len = it.w;
+      const int n_kv = (kv_len + kBN - 1) / kBN;
+      const int tok = q_start + row;
+      const float lse2 = (tok < T) ? lse[(size_t)h * T + tok] * kLog2eWs : 0.f;
+      const float dl = (tok < T) ? delta[(size_t)h * T + tok] : 0.f;
 
       for (int j = 0; j < n_kv; ++j, ++gk) {
         mbar_wait(bar(dqSFull), gk & 1, s_abort);
@@ -743,6 +746,9 @@ attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         tc_fence_before();
         mbar_arrive(bar(dqDsReady));
       }
+      // The last S and dP of this unit have been consumed, so Q/dO of the NEXT unit can move into
+      // tensor memory now; the issuing warp then starts that unit while this one's dQ is written.
+      if (snake_unit(r + 1, cta, n_cta) < n_units && !*s_abort) copy_q_do(uc + 1);
       // ---- unit epilogue: dQ rows, scaled (column groups 0 and 1 write half a row each) -----
       mbar_wait(bar(dqDone), uc & 1, s_abort);
       tc_fence_after();
