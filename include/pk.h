@@ -205,6 +205,15 @@ int pk_seqlens_from_posids_noalloc(const int32_t* position_ids, int32_t T,
                                    int32_t* max_seqlen, void* stream);
 
 /*
+ * Self-test of the bounded waits (no counterpart in the paper): one small kernel waits on a
+ * barrier that nothing will ever signal, for at most `budget_cycles` SM clocks (1 .. 2e9), then
+ * records PK_ERR_TIMEOUT (detail 99) in the status word of `workspace` (>= 128 bytes, its header
+ * must have been initialised by a planning call) and returns normally -- the same path a stuck
+ * pipeline takes inside the attention kernels.  The context stays usable.
+ */
+int pk_selftest_bounded_wait(void* workspace, int64_t budget_cycles, void* stream);
+
+/*
  * Measurement aid (no counterpart in the paper): asks the library to record the CUDA
  * events `start` and `stop` (cudaEvent_t passed as void*, owned by the caller) on the
  * call's stream immediately before and after every later launch of kernel `which`

@@ -50,6 +50,7 @@ _SIGNATURES = {
     "pk_status_read": (ctypes.c_int, [_vp, _vp, ctypes.POINTER(_i32), ctypes.POINTER(_i32)]),
     "pk_set_timing_events": (ctypes.c_int, [_i32, _vp, _vp]),
     "pk_set_rope_mode": (ctypes.c_int, [_i32]),
+    "pk_selftest_bounded_wait": (ctypes.c_int, [_vp, ctypes.c_int64, _vp]),
     "pk_seqlens_from_posids_noalloc": (ctypes.c_int, [_vp, _i32, _vp, _vp, _vp, _vp]),
 }
 
@@ -214,6 +215,11 @@ PK_ROPE_ROTATED_COPIES, PK_ROPE_IN_TILE = 0, 1
 
 def pk_set_rope_mode(mode: int) -> None:
     _check("pk_set_rope_mode", lib().pk_set_rope_mode(mode))
+
+
+def pk_selftest_bounded_wait(workspace: torch.Tensor, budget_cycles: int, stream=None) -> None:
+    _check("pk_selftest_bounded_wait",
+           lib().pk_selftest_bounded_wait(_ptr(workspace), budget_cycles, _stream(stream)))
 
 
 def workspace_view(workspace: torch.Tensor, which: int, T: int, Hq: int, Hkv: int, D: int,

@@ -1,6 +1,7 @@
 // Small host-only entry points of the C ABI: tile shape, workspace sizing and layout,
 // status read-back.
 #include "pk_common.cuh"
+#include "sm100_ptx.cuh"
 
 namespace pk {
 cudaEvent_t g_timing_events[PK_NUM_KERNELS][2] = {};
@@ -45,4 +46,33 @@ extern "C" int pk_status_read(const void* workspace, void* stream, int32_t* code
   *code = host[PK_HDR_STATUS];
   *detail = host[PK_HDR_DETAIL];
   return PK_OK;
+}
+
+namespace pk {
+namespace {
+// Waits on an mbarrier that nothing ever arrives at, with a small budget, and reports the
+// expiry through the status word exactly as the attention kernels do.
+__global__ void bounded_wait_selftest_kernel(int32_t* hdr, long long budget) {
+  __shared__ __align__(8) unsigned long long s_bar;
+  __shared__ int s_abort;
+  const uint32_t bar = ptx::smem_u32(&s_bar);
+  if (threadIdx.x == 0) {
+    ptx::mbar_init(bar, 1);
+    ptx::fence_mbar_init();
+    s_abort = 0;
+  }
+  __syncthreads();
+  const bool ok = ptx::mbar_wait_budget(bar, 0, &s_abort, budget);
+  __syncthreads();
+  if (threadIdx.x == 0 && !ok) set_status(hdr, PK_ERR_TIMEOUT, 99);
+}
+}  // namespace
+}  // namespace pk
+
+extern "C" int pk_selftest_bounded_wait(void* workspace, int64_t budget_cycles, void* stream) {
+  if (workspace == nullptr || budget_cycles <= 0 || budget_cycles > 2000000000LL)
+    return PK_ERR_INVALID_ARG;
+  pk::bounded_wait_selftest_kernel<<<1, 64, 0, static_cast<cudaStream_t>(stream)>>>(
+      static_cast<int32_t*>(workspace), (long long)budget_cycles);
+  return pk::launch_status();
 }

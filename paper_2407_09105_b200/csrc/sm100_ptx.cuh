@@ -54,17 +54,21 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 // of budget; every later wait in the CTA then returns at once so that all threads
 // drain to the common exit.  Returns false on timeout/abort.
 constexpr long long kWaitBudgetCycles = 4000000000LL;  // about two seconds
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool mbar_wait_budget(uint32_t bar, uint32_t parity,
+                                                 volatile int* abort_flag, long long budget) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   while (true) {
     if (mbar_try_wait(bar, parity)) return true;
     if (*abort_flag) return false;
-    if (clock64() - t0 > kWaitBudgetCycles) {
+    if (clock64() - t0 > budget) {
       *abort_flag = 1;
       return false;
     }
   }
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  return mbar_wait_budget(bar, parity, abort_flag, kWaitBudgetCycles);
 }
 
 __device__ __forceinline__ void fence_proxy_async_smem() {

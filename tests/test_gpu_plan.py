@@ -81,3 +81,15 @@ def test_negative_id_sets_status():
     assert code == api.PK_ERR_BAD_POSIDS and detail == 3
     hdr = api.workspace_view(ws, api.PK_WS_HEADER, 6, 1, 1, 64).cpu().numpy()
     assert hdr[api.PK_HDR_N_ITEMS] == 0
+
+
+def test_bounded_wait_expires_and_reports_timeout():
+    """A wait that nothing satisfies gives up after its budget, records PK_ERR_TIMEOUT and
+    returns; the context stays usable (the next planning call succeeds)."""
+    pos = torch.from_numpy(wl.position_ids_from_lengths([40, 9])).cuda()
+    ws, cu, ne, mx = run_plan(pos)
+    assert api.pk_status_read(ws) == (api.PK_OK, 0)
+    api.pk_selftest_bounded_wait(ws, 2_000_000)          # about a millisecond
+    assert api.pk_status_read(ws) == (api.PK_ERR_TIMEOUT, 99)
+    ws, cu, ne, mx = run_plan(pos)
+    assert api.pk_status_read(ws) == (api.PK_OK, 0) and int(ne) == 2
