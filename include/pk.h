@@ -204,6 +204,36 @@ int pk_seqlens_from_posids_noalloc(const int32_t* position_ids, int32_t T,
                                    int32_t* cu_seqlens, int32_t* n_examples,
                                    int32_t* max_seqlen, void* stream);
 
+/* ---- steps around the attention path (the scope's "next" rows) -------------------------- */
+
+/*
+ * Padding-free collator (Sec. 3.4 "PaddingFreeCollator", worked example in Sec. 3.5), on the
+ * device: the examples are already concatenated in input_ids; from their lengths it writes
+ *   cu_seqlens   int32 [E+1]  prefix sums of the lengths (cu_seqlens[0] = 0)
+ *   position_ids int32 [T]    0 .. L_e-1 for every example
+ *   labels       int32 [T]    input_ids with the first entry of every example replaced by
+ *                             ignore_index (the paper uses -100); may be NULL
+ * All pointers are device pointers.  Requires sum(lengths) == T and E >= 1 when T > 0.
+ */
+int pk_collate_padding_free(const int32_t* input_ids, const int32_t* lengths, int32_t E, int32_t T,
+                            int32_t* position_ids, int32_t* labels, int32_t* cu_seqlens,
+                            int32_t ignore_index, void* stream);
+
+/*
+ * Sample selection (Sec. 3.3), on the HOST (all pointers are host pointers): bin_of[i] receives
+ * the pack of example i, *n_bins the number of packs.  Every length must be in [1, capacity].
+ *   first_fit_decreasing  Multipack-style: examples from long to short (ties in the given
+ *                         order), each into the first pack with room
+ *   next_fit              first-come-first-served in the given order (sort_descending = 0, the
+ *                         random-order baseline) or from long to short (sort_descending = 1,
+ *                         the sorted baseline); a new pack starts when the next example does
+ *                         not fit.  Examples are never broken.
+ */
+int pk_pack_first_fit_decreasing(const int32_t* lengths, int32_t n, int32_t capacity,
+                                 int32_t* bin_of, int32_t* n_bins);
+int pk_pack_next_fit(const int32_t* lengths, int32_t n, int32_t capacity, int32_t sort_descending,
+                     int32_t* bin_of, int32_t* n_bins);
+
 /*
  * Self-test of the bounded waits (no counterpart in the paper): one small kernel waits on a
  * barrier that nothing will ever signal, for at most `budget_cycles` SM clocks (1 .. 2e9), then

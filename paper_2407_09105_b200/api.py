@@ -50,6 +50,9 @@ _SIGNATURES = {
     "pk_status_read": (ctypes.c_int, [_vp, _vp, ctypes.POINTER(_i32), ctypes.POINTER(_i32)]),
     "pk_set_timing_events": (ctypes.c_int, [_i32, _vp, _vp]),
     "pk_set_rope_mode": (ctypes.c_int, [_i32]),
+    "pk_collate_padding_free": (ctypes.c_int, [_vp, _vp, _i32, _i32, _vp, _vp, _vp, _i32, _vp]),
+    "pk_pack_first_fit_decreasing": (ctypes.c_int, [_vp, _i32, _i32, _vp, ctypes.POINTER(_i32)]),
+    "pk_pack_next_fit": (ctypes.c_int, [_vp, _i32, _i32, _i32, _vp, ctypes.POINTER(_i32)]),
     "pk_selftest_bounded_wait": (ctypes.c_int, [_vp, ctypes.c_int64, _vp]),
     "pk_seqlens_from_posids_noalloc": (ctypes.c_int, [_vp, _i32, _vp, _vp, _vp, _vp]),
 }
@@ -215,6 +218,35 @@ PK_ROPE_ROTATED_COPIES, PK_ROPE_IN_TILE = 0, 1
 
 def pk_set_rope_mode(mode: int) -> None:
     _check("pk_set_rope_mode", lib().pk_set_rope_mode(mode))
+
+
+def pk_collate_padding_free(input_ids: torch.Tensor, lengths: torch.Tensor,
+                            position_ids: torch.Tensor, labels: Optional[torch.Tensor],
+                            cu_seqlens: torch.Tensor, ignore_index: int = -100, stream=None) -> None:
+    _check("pk_collate_padding_free",
+           lib().pk_collate_padding_free(_ptr(input_ids), _ptr(lengths), lengths.numel(),
+                                         position_ids.numel(), _ptr(position_ids), _ptr(labels),
+                                         _ptr(cu_seqlens), ignore_index, _stream(stream)))
+
+
+def _pack(fn_name, lengths, capacity, *extra):
+    import numpy as np
+    arr = np.ascontiguousarray(np.asarray(lengths, dtype=np.int32))
+    out = np.empty_like(arr)
+    nb = _i32()
+    fn = getattr(lib(), fn_name)
+    _check(fn_name, fn(arr.ctypes.data, arr.size, capacity, *extra, out.ctypes.data,
+                       ctypes.byref(nb)))
+    return out.tolist(), nb.value
+
+
+def pk_pack_first_fit_decreasing(lengths, capacity: int):
+    """Host-side: (bin index per example, number of bins)."""
+    return _pack("pk_pack_first_fit_decreasing", lengths, capacity)
+
+
+def pk_pack_next_fit(lengths, capacity: int, sort_descending: bool):
+    return _pack("pk_pack_next_fit", lengths, capacity, int(sort_descending))
 
 
 def pk_selftest_bounded_wait(workspace: torch.Tensor, budget_cycles: int, stream=None) -> None:

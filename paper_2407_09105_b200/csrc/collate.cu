@@ -1,0 +1,126 @@
+// Steps around the attention path ("next" scope): the padding-free collator of Sec. 3.4 / 3.5 on
+// the device (position ids restart per example, first label of an example is ignored), and the
+// sample-selection baselines of Sec. 3.3 on the host (first-fit-decreasing as in Multipack, and
+// first-come-first-served filling).
+#include <algorithm>
+#include <numeric>
+#include <vector>
+
+#include "pk_common.cuh"
+
+namespace pk {
+namespace {
+
+// cu[0] = 0, cu[e+1] = cu[e] + lengths[e]; one CTA, chunks of 1024 examples.
+__global__ void __launch_bounds__(1024) lengths_scan_kernel(const int32_t* __restrict__ lengths,
+                                                            int E, int32_t* __restrict__ cu) {
+  __shared__ int warp_sums[33];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  int carry = 0;
+  if (tid == 0) cu[0] = 0;
+  for (int base = 0; base < E; base += 1024) {
+    const int e = base + tid;
+    const int v = e < E ? lengths[e] : 0;
+    int x = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int y = __shfl_up_sync(0xffffffffu, x, o);
+      if (lane >= o) x += y;
+    }
+    if (lane == 31) warp_sums[warp] = x;
+    __syncthreads();
+    if (warp == 0) {
+      const int w = warp_sums[lane];
+      int s = w;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int y = __shfl_up_sync(0xffffffffu, s, o);
+        if (lane >= o) s += y;
+      }
+      warp_sums[lane] = s - w;
+      if (lane == 31) warp_sums[32] = s;
+    }
+    __syncthreads();
+    if (e < E) cu[e + 1] = carry + warp_sums[warp] + x;
+    carry += warp_sums[32];
+    __syncthreads();
+  }
+}
+
+__global__ void collate_kernel(const int32_t* __restrict__ input_ids, const int32_t* __restrict__ cu,
+                               int E, int T, int32_t ignore_index, int32_t* __restrict__ position_ids,
+                               int32_t* __restrict__ labels) {
+  const int t = blockIdx.x * blockDim.x + threadIdx.x;
+  if (t >= T) return;
+  int lo = 0, hi = E - 1;                 // largest e with cu[e] <= t
+  while (lo < hi) {
+    const int mid = (lo + hi + 1) >> 1;
+    if (cu[mid] <= t) lo = mid; else hi = mid - 1;
+  }
+  const int p = t - cu[lo];
+  position_ids[t] = p;
+  if (labels != nullptr) labels[t] = (p == 0) ? ignore_index : input_ids[t];
+}
+
+}  // namespace
+}  // namespace pk
+
+extern "C" int pk_collate_padding_free(const int32_t* input_ids, const int32_t* lengths, int32_t E,
+                                       int32_t T, int32_t* position_ids, int32_t* labels,
+                                       int32_t* cu_seqlens, int32_t ignore_index, void* stream_) {
+  if (E < 0 || T < 0 || cu_seqlens == nullptr) return PK_ERR_INVALID_ARG;
+  if ((E > 0 && lengths == nullptr) || (T > 0 && position_ids == nullptr)) return PK_ERR_INVALID_ARG;
+  if (T > 0 && (E == 0 || (labels != nullptr && input_ids == nullptr))) return PK_ERR_INVALID_ARG;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  pk::lengths_scan_kernel<<<1, 1024, 0, stream>>>(lengths, E, cu_seqlens);
+  if (pk::launch_status() != PK_OK) return PK_ERR_CUDA;
+  if (T == 0) return PK_OK;
+  pk::collate_kernel<<<(T + 255) / 256, 256, 0, stream>>>(input_ids, cu_seqlens, E, T, ignore_index,
+                                                         position_ids, labels);
+  return pk::launch_status();
+}
+
+extern "C" int pk_pack_first_fit_decreasing(const int32_t* lengths, int32_t n, int32_t capacity,
+                                            int32_t* bin_of, int32_t* n_bins) {
+  if (n < 0 || capacity <= 0 || n_bins == nullptr || (n > 0 && (!lengths || !bin_of)))
+    return PK_ERR_INVALID_ARG;
+  for (int i = 0; i < n; ++i)
+    if (lengths[i] <= 0 || lengths[i] > capacity) return PK_ERR_INVALID_ARG;
+  std::vector<int32_t> order(n);
+  std::iota(order.begin(), order.end(), 0);
+  std::stable_sort(order.begin(), order.end(),
+                   [&](int32_t a, int32_t b) { return lengths[a] > lengths[b]; });
+  std::vector<int32_t> room;
+  for (int32_t i : order) {
+    size_t b = 0;
+    while (b < room.size() && room[b] < lengths[i]) ++b;
+    if (b == room.size()) room.push_back(capacity);
+    room[b] -= lengths[i];
+    bin_of[i] = (int32_t)b;
+  }
+  *n_bins = (int32_t)room.size();
+  return PK_OK;
+}
+
+extern "C" int pk_pack_next_fit(const int32_t* lengths, int32_t n, int32_t capacity,
+                                int32_t sort_descending, int32_t* bin_of, int32_t* n_bins) {
+  if (n < 0 || capacity <= 0 || n_bins == nullptr || (n > 0 && (!lengths || !bin_of)))
+    return PK_ERR_INVALID_ARG;
+  for (int i = 0; i < n; ++i)
+    if (lengths[i] <= 0 || lengths[i] > capacity) return PK_ERR_INVALID_ARG;
+  std::vector<int32_t> order(n);
+  std::iota(order.begin(), order.end(), 0);
+  if (sort_descending)
+    std::stable_sort(order.begin(), order.end(),
+                     [&](int32_t a, int32_t b) { return lengths[a] > lengths[b]; });
+  int32_t b = 0, used = 0;
+  bool started = false;
+  for (int32_t i : order) {
+    if (started && used + lengths[i] > capacity) { ++b; used = 0; }
+    bin_of[i] = b;
+    used += lengths[i];
+    started = true;
+  }
+  *n_bins = started ? b + 1 : 0;
+  return PK_OK;
+}
