@@ -43,7 +43,7 @@ constexpr int kCW = 128 / kNQ;                            // columns per compute
 constexpr int kWsThreads = kComputeThreads + 64;
 constexpr int kMmaWarp = kComputeThreads / 32;
 constexpr int kLoadWarp = kMmaWarp + 1;
-static_assert(kNQ == 2, "the dK/dV kernel assigns two 32-column pieces per compute thread");
+static_assert(kNQ == 2, "the dK/dV kernel gives each compute thread 64 query columns");
 constexpr float kLog2eWs = 1.4426950408889634f;
 
 // position in the longest-first order of the r-th unit of this CTA (snake over the rounds)
@@ -62,23 +62,32 @@ struct DkvSmem {
   static constexpr int kBoxBytes = 128 * 128;
   static constexpr int kBoxes = D / 64;
   static constexpr int kTileBytes = kBoxBytes * kBoxes;
+  static constexpr int kQStages = 3;                         // Q is needed until dK of its step
+  static constexpr int kDoStages = 2;
   static constexpr int kK = 0;
   static constexpr int kV = kTileBytes;
-  static constexpr int kQ0 = 2 * kTileBytes;                 // stage s: Q at kQ0 + s*2*tile
-  static constexpr int kStageBytes = 2 * kTileBytes;         // Q then dO
-  static constexpr int kdS = kQ0 + 2 * kStageBytes;          // 2 boxes
-  static constexpr int kLse = kdS + 2 * kBoxBytes;           // [2][128] floats
+  static constexpr int kQ0 = 2 * kTileBytes;                 // Q ring
+  static constexpr int kDo0 = kQ0 + kQStages * kTileBytes;   // dO ring
+  static constexpr int kLse = kDo0 + kDoStages * kTileBytes; // [2][128] floats, slot = step & 1
   static constexpr int kDelta = kLse + 1024;                 // [2][128] floats
   static constexpr int kBars = kDelta + 1024;
-  static constexpr int kMisc = kBars + 16 * 8;
+  static constexpr int kMisc = kBars + 24 * 8;
   static constexpr int kTotal = kMisc + 16;
 };
 
 enum DkvBar {
-  kvKvFull = 0, kvKvEmpty, kvQFull0, kvQFull1, kvDoFull0, kvDoFull1, kvQdoEmpty0, kvQdoEmpty1,
-  kvSFull, kvDpFull, kvPReady, kvPReadyA, kvDsReady, kvUnitDone, kvDkvRead, kvNumBars
+  kvKvFull = 0, kvKvEmpty,
+  kvQFull0, kvQFull1, kvQFull2, kvDoFull0, kvDoFull1, kvQEmpty0, kvQEmpty1, kvQEmpty2,
+  kvSFull, kvDpFull, kvPReady, kvDsReady, kvDpRead, kvUnitDone, kvDkvRead, kvNumBars
 };
+static_assert(kvNumBars <= 24, "barrier area");
 
+// Tensor memory of the dK/dV kernel: two 128-column regions that trade roles every step, then
+// the dV and dK accumulators.  Step n keeps S^T in region n & 1; each compute thread overwrites
+// its own 64 columns of it with P^T (first 32 columns, 64 bf16) and dS^T (last 32), so no thread
+// ever writes a column another thread still has to read.  dP^T of step n sits in the other
+// region, and S^T of step n+1 is written there as soon as every thread holds dP^T(n) in
+// registers: the next step's scores never wait for the tensor pipe to consume P^T or dS^T.
 template <int D, bool kRot, typename GradT>
 __global__ void __launch_bounds__(kWsThreads, 1)
 attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
@@ -91,7 +100,7 @@ attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   using L = DkvSmem<D>;
   extern __shared__ __align__(1024) uint8_t smem[];
   const uint32_t sbase = smem_u32(smem);
-  const uint32_t sK = sbase + L::kK, sV = sbase + L::kV, sdS = sbase + L::kdS;
+  const uint32_t sK = sbase + L::kK, sV = sbase + L::kV;
   float* s_lse = reinterpret_cast<float*>(smem + L::kLse);
   float* s_delta = reinterpret_cast<float*>(smem + L::kDelta);
   const uint32_t bars = sbase + L::kBars;
@@ -104,17 +113,16 @@ attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   if (tid == 0) {
     mbar_init(bar(kvKvFull), 1);
     mbar_init(bar(kvKvEmpty), 1);
-    mbar_init(bar(kvQFull0), 33);
-    mbar_init(bar(kvQFull1), 33);
-    mbar_init(bar(kvDoFull0), 1);
-    mbar_init(bar(kvDoFull1), 1);
-    mbar_init(bar(kvQdoEmpty0), 1);
-    mbar_init(bar(kvQdoEmpty1), 1);
+    for (int i = 0; i < L::kQStages; ++i) {
+      mbar_init(bar(kvQFull0 + i), 1);
+      mbar_init(bar(kvQEmpty0 + i), 1);
+    }
+    for (int i = 0; i < L::kDoStages; ++i) mbar_init(bar(kvDoFull0 + i), 33);
     mbar_init(bar(kvSFull), 1);
     mbar_init(bar(kvDpFull), 1);
     mbar_init(bar(kvPReady), kComputeThreads);
-    mbar_init(bar(kvPReadyA), kComputeThreads);
     mbar_init(bar(kvDsReady), kComputeThreads);
+    mbar_init(bar(kvDpRead), kComputeThreads);
     mbar_init(bar(kvUnitDone), 1);
     mbar_init(bar(kvDkvRead), kComputeThreads);
     fence_mbar_init();
@@ -128,7 +136,9 @@ attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = static_cast<uint32_t>(*s_tmem);
-  const uint32_t tS = tmem, tdP = tmem + 128, tdV = tmem + 256, tdK = tmem + 384;
+  const uint32_t tdV = tmem + 256, tdK = tmem + 384;
+  auto region_s = [&](int n) { return tmem + static_cast<uint32_t>(n & 1) * 128u; };
+  auto region_dp = [&](int n) { return tmem + static_cast<uint32_t>((n & 1) ^ 1) * 128u; };
 
   const int G = Hq / Hkv;
   const bool plan_ok = (hdr[PK_HDR_PLAN_T] == T);
@@ -138,6 +148,10 @@ attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 
   if (warp == kLoadWarp) {
     // =============================== loader ===============================================
+    // Steps are numbered globally (gs) across this CTA's units.  Q(gs) goes to Q stage gs % 3 once
+    // dK of step gs-3 has retired; dO(gs) and the lse / delta rows go to slot gs & 1 once dK of step
+    // gs-2 has retired (dV(gs-2) precedes it on the tensor pipe, and the compute warps are done
+    // with that step's lse / delta before they hand over its dS).
     if (lane == 0) {
       prefetch_tensormap(&tm_q);
       prefetch_tensormap(&tm_k);
@@ -164,35 +178,43 @@ attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       for (int hh = 0; hh < G; ++hh) {
         const int h = g * G + hh;
         for (int i = 0; i < n_q; ++i, ++gs) {
-          const int st = gs & 1;
+          const int qs = gs % L::kQStages, sl = gs & 1;
           const int q0 = q_start + i * kBM;
-          mbar_wait(bar(kvQdoEmpty0 + st), ((gs >> 1) & 1) ^ 1, s_abort);
-          const uint32_t sQ = sbase + L::kQ0 + st * L::kStageBytes, sdO = sQ + L::kTileBytes;
+          mbar_wait(bar(kvQEmpty0 + qs), ((gs / L::kQStages) & 1) ^ 1, s_abort);
           if (lane == 0) {
-            mbar_expect_tx(bar(kvQFull0 + st), L::kTileBytes);
+            const uint32_t sQ = sbase + L::kQ0 + qs * L::kTileBytes;
+            mbar_expect_tx(bar(kvQFull0 + qs), L::kTileBytes);
 #pragma unroll
             for (int b = 0; b < L::kBoxes; ++b)
-              tma_load_2d(sQ + b * L::kBoxBytes, &tm_q, h * D + b * 64, q0, bar(kvQFull0 + st));
-            mbar_expect_tx(bar(kvDoFull0 + st), L::kTileBytes);
+              tma_load_2d(sQ + b * L::kBoxBytes, &tm_q, h * D + b * 64, q0, bar(kvQFull0 + qs));
+          }
+          if (gs >= 2) {
+            const int e = gs - 2;
+            mbar_wait(bar(kvQEmpty0 + e % L::kQStages), (e / L::kQStages) & 1, s_abort);
+          }
+          if (lane == 0) {
+            const uint32_t sdO = sbase + L::kDo0 + sl * L::kTileBytes;
+            mbar_expect_tx(bar(kvDoFull0 + sl), L::kTileBytes);
 #pragma unroll
             for (int b = 0; b < L::kBoxes; ++b)
-              tma_load_2d(sdO + b * L::kBoxBytes, &tm_do, h * D + b * 64, q0, bar(kvDoFull0 + st));
+              tma_load_2d(sdO + b * L::kBoxBytes, &tm_do, h * D + b * 64, q0, bar(kvDoFull0 + sl));
           }
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
             const int row = lane * 4 + e, tok = q0 + row;
             const bool in = tok < T;
-            s_lse[st * 128 + row] = in ? lse[(size_t)h * T + tok] * kLog2eWs : 0.f;
-            s_delta[st * 128 + row] = in ? delta[(size_t)h * T + tok] : 0.f;
+            s_lse[sl * 128 + row] = in ? lse[(size_t)h * T + tok] * kLog2eWs : 0.f;
+            s_delta[sl * 128 + row] = in ? delta[(size_t)h * T + tok] : 0.f;
           }
-          mbar_arrive(bar(kvQFull0 + st));
+          mbar_arrive(bar(kvDoFull0 + sl));
         }
       }
     }
   } else if (warp == kMmaWarp) {
     // =============================== MMA issuer ===========================================
     // The whole warp walks the schedule (so that addresses and descriptors stay warp-uniform);
-    // one elected lane issues the tensor-core instructions.
+    // one elected lane issues the tensor-core instructions.  Per step, in tensor-pipe order:
+    //   S^T(s+1) | dV += P^T(s) dO | dK += dS^T(s) Q | dP^T(s+1)
     {
       // kRot: q and k are the rotated fp16 copies; dS then follows their format (operands of one
       // contraction must share a format), everything touching V, dO and P stays bf16
@@ -202,27 +224,35 @@ attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       constexpr uint32_t kIdescDV = make_idesc(128, D, kFmtBF16, kFmtBF16, 0, 1);
       constexpr uint32_t kIdescDK = make_idesc(128, D, kQKFmt, kQKFmt, 0, 1);
       const bool leader = elect_one();
-      const uint32_t k_lo = desc_lo(sK, 16), v_lo = desc_lo(sV, 16), ds_lo = desc_lo(sdS, 16);
+      const uint32_t k_lo = desc_lo(sK, 16), v_lo = desc_lo(sV, 16);
       int gs = 0, uc = 0;
-      auto issue_s = [&](int st) {
-        const uint32_t q_lo = desc_lo(sbase + L::kQ0 + st * L::kStageBytes, 16);
+      auto issue_s = [&](int n) {   // S^T(n) = K Q(n)^T into region_s(n)
+        const int qs = n % L::kQStages;
+        mbar_wait(bar(kvQFull0 + qs), (n / L::kQStages) & 1, s_abort);
+        tc_fence_after();
+        const uint32_t q_lo = desc_lo(sbase + L::kQ0 + qs * L::kTileBytes, 16);
+        const uint32_t dst = region_s(n);
         if (leader) {
 #pragma unroll
           for (int kk = 0; kk < D / 16; ++kk) {
             const uint32_t off = ((kk / 4) * L::kBoxBytes + (kk % 4) * 32) >> 4;
-            mma_ss(tS, desc_from_lo(k_lo + off), desc_from_lo(q_lo + off), kIdescS, kk > 0);
+            mma_ss(dst, desc_from_lo(k_lo + off), desc_from_lo(q_lo + off), kIdescS, kk > 0);
           }
           mma_commit(bar(kvSFull));
         }
         __syncwarp();
       };
-      auto issue_dp = [&](int st) {
-        const uint32_t do_lo = desc_lo(sbase + L::kQ0 + st * L::kStageBytes + L::kTileBytes, 16);
+      auto issue_dp = [&](int n) {  // dP^T(n) = V dO(n)^T into region_dp(n)
+        const int sl = n & 1;
+        mbar_wait(bar(kvDoFull0 + sl), (n >> 1) & 1, s_abort);
+        tc_fence_after();
+        const uint32_t do_lo = desc_lo(sbase + L::kDo0 + sl * L::kTileBytes, 16);
+        const uint32_t dst = region_dp(n);
         if (leader) {
 #pragma unroll
           for (int kk = 0; kk < D / 16; ++kk) {
             const uint32_t off = ((kk / 4) * L::kBoxBytes + (kk % 4) * 32) >> 4;
-            mma_ss(tdP, desc_from_lo(v_lo + off), desc_from_lo(do_lo + off), kIdescDP, kk > 0);
+            mma_ss(dst, desc_from_lo(v_lo + off), desc_from_lo(do_lo + off), kIdescDP, kk > 0);
           }
           mma_commit(bar(kvDpFull));
         }
@@ -235,62 +265,51 @@ attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         const int n_q = (it.w + kBM - 1) / kBM;
         const int n_steps = G * n_q;
         mbar_wait(bar(kvKvFull), uc & 1, s_abort);
-        // prologue: S(0), dP(0).  The compute warps finished reading S and dP of the previous
-        // unit's last step before they signalled its dS, which the last dK waited for.
-        mbar_wait(bar(kvQFull0 + (gs & 1)), (gs >> 1) & 1, s_abort);
+        // prologue: S(0) goes where dP of the previous unit's last step was, so that one must
+        // have been read; dP(0) goes where P / dS of that step were, which its dV / dK consumed
+        // earlier on the tensor pipe
+        if (gs > 0) mbar_wait(bar(kvDpRead), (gs - 1) & 1, s_abort);
         tc_fence_after();
-        issue_s(gs & 1);
-        mbar_wait(bar(kvDoFull0 + (gs & 1)), (gs >> 1) & 1, s_abort);
-        tc_fence_after();
-        issue_dp(gs & 1);
+        issue_s(gs);
+        issue_dp(gs);
         for (int s = 0; s < n_steps; ++s, ++gs) {
-          const int st = gs & 1;
-          const uint32_t stage = sbase + L::kQ0 + st * L::kStageBytes;
-          const uint32_t qT_lo = desc_lo(stage, L::kBoxBytes);                      // Q, MN-major
-          const uint32_t doT_lo = desc_lo(stage + L::kTileBytes, L::kBoxBytes);     // dO, MN-major
+          const uint32_t tA = region_s(gs);
+          const uint32_t doT_lo = desc_lo(sbase + L::kDo0 + (gs & 1) * L::kTileBytes, L::kBoxBytes);
+          const uint32_t qT_lo =
+              desc_lo(sbase + L::kQ0 + (gs % L::kQStages) * L::kTileBytes, L::kBoxBytes);
           const uint32_t acc = s > 0 ? 1u : 0u;
-          mbar_wait(bar(kvPReadyA), gs & 1, s_abort);   // first 64 query columns of P
+          const bool more = (s + 1 < n_steps);
+          if (more) {                             // S(s+1) over dP(s), which sits in registers now
+            // (the TMA barrier first: it completed long ago, and polling it costs time best
+            // spent while dP(s) is still being read)
+            mbar_wait(bar(kvQFull0 + (gs + 1) % L::kQStages), ((gs + 1) / L::kQStages) & 1, s_abort);
+            mbar_wait(bar(kvDpRead), gs & 1, s_abort);
+            tc_fence_after();
+            issue_s(gs + 1);
+          } else {
+            mbar_wait(bar(kvPReady), gs & 1, s_abort);
+          }
+          // every thread hands over P^T before it reads dP^T, so the wait above covers P^T as well
           if (s == 0 && uc > 0) mbar_wait(bar(kvDkvRead), (uc - 1) & 1, s_abort);
           tc_fence_after();
           if (leader) {
 #pragma unroll
-            for (int kk = 0; kk < kBM / 32; ++kk)   // dV += P^T dO, first half of the query rows
-              mma_ts(tdV, tS + kk * 8, desc_from_lo(doT_lo + ((kk * 2048) >> 4)), kIdescDV,
-                     acc | (kk > 0));
+            for (int kk = 0; kk < kBM / 16; ++kk)   // dV += P^T dO; P^T of queries 16kk.. : see compute
+              mma_ts(tdV, tA + (kk / 4) * 64 + (kk % 4) * 8, desc_from_lo(doT_lo + ((kk * 2048) >> 4)),
+                     kIdescDV, acc | (kk > 0));
           }
           __syncwarp();
-          mbar_wait(bar(kvPReady), gs & 1, s_abort);    // second half
-          tc_fence_after();
-          if (leader) {
-#pragma unroll
-            for (int kk = kBM / 32; kk < kBM / 16; ++kk)
-              mma_ts(tdV, tS + kk * 8, desc_from_lo(doT_lo + ((kk * 2048) >> 4)), kIdescDV, 1u);
-          }
-          __syncwarp();
-          const bool more = (s + 1 < n_steps);
-          const int g1 = gs + 1;
-          if (more) {                              // S(s+1): P(s) was consumed by dV(s) above
-            mbar_wait(bar(kvQFull0 + (g1 & 1)), (g1 >> 1) & 1, s_abort);
-            tc_fence_after();
-            issue_s(g1 & 1);
-          }
           mbar_wait(bar(kvDsReady), gs & 1, s_abort);
           tc_fence_after();
           if (leader) {
 #pragma unroll
-            for (int kk = 0; kk < kBM / 16; ++kk) {   // dK += dS^T Q
-              const uint32_t off = ((kk / 4) * L::kBoxBytes + (kk % 4) * 32) >> 4;
-              mma_ss(tdK, desc_from_lo(ds_lo + off), desc_from_lo(qT_lo + ((kk * 2048) >> 4)),
-                     kIdescDK, acc | (kk > 0));
-            }
-            mma_commit(bar(kvQdoEmpty0 + st));
+            for (int kk = 0; kk < kBM / 16; ++kk)   // dK += dS^T Q
+              mma_ts(tdK, tA + (kk / 4) * 64 + 32 + (kk % 4) * 8,
+                     desc_from_lo(qT_lo + ((kk * 2048) >> 4)), kIdescDK, acc | (kk > 0));
+            mma_commit(bar(kvQEmpty0 + gs % L::kQStages));
           }
           __syncwarp();
-          if (more) {                              // dP(s+1): dP(s) was read before dS(s) was signalled
-            mbar_wait(bar(kvDoFull0 + (g1 & 1)), (g1 >> 1) & 1, s_abort);
-            tc_fence_after();
-            issue_dp(g1 & 1);
-          }
+          if (more) issue_dp(gs + 1);             // over P / dS(s), consumed just above
         }
         if (leader) {
           mma_commit(bar(kvUnitDone));
@@ -302,8 +321,9 @@ attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   } else {
     // =============================== compute ===============================================
     const int row = tid & 127;              // key row inside the block
-    const int qd = tid >> 7;                // which group of kCW query columns
+    const int qd = tid >> 7;                // this thread's query columns: [64*qd, +64)
     const uint32_t lane_off = static_cast<uint32_t>((warp & 3) * 32) << 16;
+    const int col0 = qd * kCW;
     int gs = 0, uc = 0;
     for (int r = 0;; ++r, ++uc) {
       const int u = snake_unit(r, cta, n_cta);
@@ -314,85 +334,70 @@ attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       const int n_q = (q_len + kBM - 1) / kBM;
       for (int hh = 0; hh < G; ++hh) {
         for (int i = 0; i < n_q; ++i, ++gs) {
-          const int st = gs & 1;
+          const int sl = gs & 1;
           const int q_left = q_len - i * kBM;
           const int col_min = (i == 0) ? row : 0;
-          // This thread's 64 query columns are taken in two pieces, [32*qd, +32) of the first 64
-          // and of the second 64, so that all warps finish the first half of P together and dV
-          // can start on it while the second half is still being exponentiated.
-          const int col_a = qd * 32, col_b = 64 + qd * 32;
-          mbar_wait(bar(kvQFull0 + st), (gs >> 1) & 1, s_abort);   // lse / delta rows visible
+          const uint32_t tA = region_s(gs) + lane_off + col0;    // S^T, then P^T | dS^T
+          const uint32_t tB = region_dp(gs) + lane_off + col0;   // dP^T
+          mbar_wait(bar(kvDoFull0 + sl), (gs >> 1) & 1, s_abort);   // lse / delta rows visible
           mbar_wait(bar(kvSFull), gs & 1, s_abort);
           tc_fence_after();
           float p[64];
-          uint32_t sv[64];
-          tmem_ld32(tS + lane_off + col_a, sv);
-          tmem_ld32(tS + lane_off + col_b, sv + 32);
-          tmem_wait_ld();
-          const bool edge = (i == 0 || q_left < kBM);   // diagonal tile or last, partial tile
+          {
+            uint32_t sv[64];
+            tmem_ld32(tA, sv);
+            tmem_ld32(tA + 32, sv + 32);
+            tmem_wait_ld();
+            const float4* lse4 = reinterpret_cast<const float4*>(s_lse + sl * 128 + col0);
 #pragma unroll
-          for (int half = 0; half < 2; ++half) {
-            const int col0 = half == 0 ? col_a : col_b;
-            const float4* lse4 = reinterpret_cast<const float4*>(s_lse + st * 128 + col0);
-#pragma unroll
-            for (int c = 0; c < 32; c += 4) {
+            for (int c = 0; c < 64; c += 4) {
               const float4 l4 = lse4[c >> 2];
-              const int k = half * 32 + c;
-              p[k] = fast_exp2(fmaf(__uint_as_float(sv[k]), scale_log2, -l4.x));
-              p[k + 1] = fast_exp2(fmaf(__uint_as_float(sv[k + 1]), scale_log2, -l4.y));
-              p[k + 2] = fast_exp2(fmaf(__uint_as_float(sv[k + 2]), scale_log2, -l4.z));
-              p[k + 3] = fast_exp2(fmaf(__uint_as_float(sv[k + 3]), scale_log2, -l4.w));
+              p[c] = fast_exp2(fmaf(__uint_as_float(sv[c]), scale_log2, -l4.x));
+              p[c + 1] = fast_exp2(fmaf(__uint_as_float(sv[c + 1]), scale_log2, -l4.y));
+              p[c + 2] = fast_exp2(fmaf(__uint_as_float(sv[c + 2]), scale_log2, -l4.z));
+              p[c + 3] = fast_exp2(fmaf(__uint_as_float(sv[c + 3]), scale_log2, -l4.w));
             }
-            if (edge) {   // interior tiles skip the compares
-#pragma unroll
-              for (int c = 0; c < 32; ++c) {
-                const int col = col0 + c;
-                if (!((col >= col_min) && (col < q_left))) p[half * 32 + c] = 0.f;
-              }
-            }
-            if (half == 0) {   // every thread has loaded S: P may overwrite its columns
-              tc_fence_before();
-              compute_bar_sync();
-              tc_fence_after();
-            }
-            uint32_t pp[16];
-#pragma unroll
-            for (int c = 0; c < 16; ++c) pp[c] = pack_bf16x2(p[half * 32 + 2 * c], p[half * 32 + 2 * c + 1]);
-            tmem_st16(tS + lane_off + half * 32 + qd * 16, pp);
-            tmem_wait_st();
-            tc_fence_before();
-            mbar_arrive(bar(half == 0 ? kvPReadyA : kvPReady));
           }
+          if (i == 0 || q_left < kBM) {   // diagonal tile or last, partial tile; interior tiles skip this
+#pragma unroll
+            for (int c = 0; c < 64; ++c) {
+              const int col = col0 + c;
+              if (!((col >= col_min) && (col < q_left))) p[c] = 0.f;
+            }
+          }
+          {
+            uint32_t pp[32];
+#pragma unroll
+            for (int c = 0; c < 32; ++c) pp[c] = pack_bf16x2(p[2 * c], p[2 * c + 1]);
+            tmem_st32(tA, pp);            // over this thread's own S^T columns
+          }
+          tmem_wait_st();
+          tc_fence_before();
+          mbar_arrive(bar(kvPReady));
 
           mbar_wait(bar(kvDpFull), gs & 1, s_abort);
           tc_fence_after();
-#pragma unroll
-          for (int c2 = 0; c2 < 2; ++c2) {
-            const int col0 = c2 == 0 ? col_a : col_b;
-            // dS^T row `row`, query columns [col0, +32): box c2, 16-byte chunks 4*qd .. 4*qd+3
-            uint8_t* ds_row = smem + L::kdS + c2 * L::kBoxBytes + row * 128;
-            const float4* dl4 = reinterpret_cast<const float4*>(s_delta + st * 128 + col0);
-            uint32_t dp[32], dd[16];
-            tmem_ld32(tdP + lane_off + col0, dp);
+          {
+            uint32_t dp[64], dd[32];
+            tmem_ld32(tB, dp);
+            tmem_ld32(tB + 32, dp + 32);
             tmem_wait_ld();
+            tc_fence_before();
+            mbar_arrive(bar(kvDpRead));   // the next S^T may be written over dP^T
+            const float4* dl4 = reinterpret_cast<const float4*>(s_delta + sl * 128 + col0);
 #pragma unroll
-            for (int e = 0; e < 32; e += 4) {
+            for (int e = 0; e < 64; e += 4) {
               const float4 d4 = dl4[e >> 2];
-              const float d0 = p[c2 * 32 + e] * (__uint_as_float(dp[e]) - d4.x);
-              const float d1 = p[c2 * 32 + e + 1] * (__uint_as_float(dp[e + 1]) - d4.y);
-              const float d2 = p[c2 * 32 + e + 2] * (__uint_as_float(dp[e + 2]) - d4.z);
-              const float d3 = p[c2 * 32 + e + 3] * (__uint_as_float(dp[e + 3]) - d4.w);
+              const float d0 = p[e] * (__uint_as_float(dp[e]) - d4.x);
+              const float d1 = p[e + 1] * (__uint_as_float(dp[e + 1]) - d4.y);
+              const float d2 = p[e + 2] * (__uint_as_float(dp[e + 2]) - d4.z);
+              const float d3 = p[e + 3] * (__uint_as_float(dp[e + 3]) - d4.w);
               dd[e >> 1] = kRot ? pack_f16x2(d0, d1) : pack_bf16x2(d0, d1);
               dd[(e >> 1) + 1] = kRot ? pack_f16x2(d2, d3) : pack_bf16x2(d2, d3);
             }
-#pragma unroll
-            for (int ch = 0; ch < 4; ++ch) {
-              const int chunk = (qd * 4 + ch) ^ (row & 7);
-              *reinterpret_cast<uint4*>(ds_row + (chunk << 4)) =
-                  make_uint4(dd[ch * 4], dd[ch * 4 + 1], dd[ch * 4 + 2], dd[ch * 4 + 3]);
-            }
+            tmem_st32(tA + 32, dd);
           }
-          fence_proxy_async_smem();
+          tmem_wait_st();
           tc_fence_before();
           mbar_arrive(bar(kvDsReady));
         }
