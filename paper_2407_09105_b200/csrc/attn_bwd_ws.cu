@@ -19,8 +19,7 @@
 // the rows of lane quarter w%4; 16 warps of 32 columns measured slightly slower because they
 // take issue slots from the warp that feeds the tensor pipe), one warp that walks the MMA
 // schedule with one elected lane issuing every tcgen05.mma, one warp that drives TMA.
-// Units are assigned statically: CTA c takes positions c, 2P-1-c, 2P+c, ... of the plan's
-// longest-first order, so the roles enumerate the same sequence without talking to each other.
+// Units are drawn from a counter (see kUnitRing below) in the plan's order.
 // Every wait is bounded; on expiry an abort flag makes all later waits return at once.
 #include <cuda_bf16.h>
 
@@ -46,10 +45,16 @@ constexpr int kLoadWarp = kMmaWarp + 1;
 static_assert(kNQ == 2, "the dK/dV kernel gives each compute thread 64 query columns");
 constexpr float kLog2eWs = 1.4426950408889634f;
 
-// position in the longest-first order of the r-th unit of this CTA (snake over the rounds)
-__device__ __forceinline__ int snake_unit(int r, int cta, int n_cta) {
-  return r * n_cta + ((r & 1) ? (n_cta - 1 - cta) : cta);
-}
+// Units are handed out dynamically: the TMA warp draws the next position of the plan's order
+// from a counter in the workspace header and publishes it to the other roles through a small
+// ring in shared memory (one mbarrier per slot).  The order keeps the units of an example next
+// to each other, so the CTAs that run at the same time share tiles in L2, and drawing from it
+// keeps every CTA busy to the end (dealt out statically, the slowest CTA of the dK/dV kernel
+// carried a fifth more steps than the mean on 8k-token packs).  A slot is rewritten four units
+// later; no role can fall that far behind the TMA warp, which waits for the previous unit's
+// tiles to be released before it loads the next one's.
+constexpr int kUnitRing = 4;
+
 __device__ __forceinline__ void compute_bar_sync() {
   asm volatile("bar.sync 1, %0;" ::"n"(kComputeThreads) : "memory");
 }
@@ -71,14 +76,15 @@ struct DkvSmem {
   static constexpr int kLse = kDo0 + kDoStages * kTileBytes; // [2][128] floats, slot = step & 1
   static constexpr int kDelta = kLse + 1024;                 // [2][128] floats
   static constexpr int kBars = kDelta + 1024;
-  static constexpr int kMisc = kBars + 24 * 8;
-  static constexpr int kTotal = kMisc + 16;
+  static constexpr int kMisc = kBars + 24 * 8;               // tmem base, abort flag, unit ring
+  static constexpr int kTotal = kMisc + 16 + 4 * kUnitRing;
 };
 
 enum DkvBar {
   kvKvFull = 0, kvKvEmpty,
   kvQFull0, kvQFull1, kvQFull2, kvDoFull0, kvDoFull1, kvQEmpty0, kvQEmpty1, kvQEmpty2,
-  kvSFull, kvDpFull, kvPReady, kvDsReady, kvDpRead, kvUnitDone, kvDkvRead, kvNumBars
+  kvSFull, kvDpFull, kvPReady, kvDsReady, kvDpRead, kvUnitDone, kvDkvRead,
+  kvUnitFull0, kvUnitFull1, kvUnitFull2, kvUnitFull3, kvNumBars
 };
 static_assert(kvNumBars <= 24, "barrier area");
 
@@ -107,6 +113,7 @@ attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   auto bar = [&](int i) { return bars + 8u * (uint32_t)i; };
   volatile int* s_tmem = reinterpret_cast<volatile int*>(smem + L::kMisc);
   volatile int* s_abort = s_tmem + 1;
+  volatile int* s_unit = s_tmem + 4;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
@@ -125,6 +132,7 @@ attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     mbar_init(bar(kvDpRead), kComputeThreads);
     mbar_init(bar(kvUnitDone), 1);
     mbar_init(bar(kvDkvRead), kComputeThreads);
+    for (int i = 0; i < kUnitRing; ++i) mbar_init(bar(kvUnitFull0 + i), 1);
     fence_mbar_init();
     *s_abort = ((sbase & 1023u) != 0) ? 1 : 0;   // swizzled tiles need a 1024-byte aligned base
   }
@@ -144,7 +152,6 @@ attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   const bool plan_ok = (hdr[PK_HDR_PLAN_T] == T);
   if (!plan_ok && blockIdx.x == 0 && tid == 0) set_status(hdr, PK_ERR_NO_PLAN, T);
   const int n_units = plan_ok ? hdr[PK_HDR_N_ITEMS] * Hkv : 0;
-  const int n_cta = gridDim.x, cta = blockIdx.x;
 
   if (warp == kLoadWarp) {
     // =============================== loader ===============================================
@@ -159,8 +166,14 @@ attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       prefetch_tensormap(&tm_do);
     }
     int gs = 0, uc = 0;
-    for (int r = 0;; ++r, ++uc) {
-      const int u = snake_unit(r, cta, n_cta);
+    for (;; ++uc) {
+      int u = 0;
+      if (lane == 0) {
+        u = atomicAdd(&hdr[kHdrBwdTicket], 1);
+        s_unit[uc % kUnitRing] = u;
+        mbar_arrive(bar(kvUnitFull0 + uc % kUnitRing));
+      }
+      u = __shfl_sync(0xffffffffu, u, 0);
       if (u >= n_units || *s_abort) break;
       const int4 it = items[order[u / Hkv]];
       const int g = u % Hkv;
@@ -258,8 +271,9 @@ attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         }
         __syncwarp();
       };
-      for (int r = 0;; ++r, ++uc) {
-        const int u = snake_unit(r, cta, n_cta);
+      for (;; ++uc) {
+        mbar_wait(bar(kvUnitFull0 + uc % kUnitRing), (uc / kUnitRing) & 1, s_abort);
+        const int u = s_unit[uc % kUnitRing];
         if (u >= n_units || *s_abort) break;
         const int4 it = items[order[u / Hkv]];
         const int n_q = (it.w + kBM - 1) / kBM;
@@ -325,8 +339,9 @@ attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     const uint32_t lane_off = static_cast<uint32_t>((warp & 3) * 32) << 16;
     const int col0 = qd * kCW;
     int gs = 0, uc = 0;
-    for (int r = 0;; ++r, ++uc) {
-      const int u = snake_unit(r, cta, n_cta);
+    for (;; ++uc) {
+      mbar_wait(bar(kvUnitFull0 + uc % kUnitRing), (uc / kUnitRing) & 1, s_abort);
+      const int u = s_unit[uc % kUnitRing];
       if (u >= n_units || *s_abort) break;
       const int4 it = items[order[u / Hkv]];
       const int g = u % Hkv;
@@ -479,14 +494,14 @@ struct DqSmem {
   static constexpr int kK0 = 2 * kTileBytes;
   static constexpr int kV0 = kK0 + kKStages * kTileBytes;
   static constexpr int kBars = kV0 + kVStages * kTileBytes;
-  static constexpr int kMisc = kBars + 24 * 8;
-  static constexpr int kTotal = kMisc + 16;
+  static constexpr int kMisc = kBars + 24 * 8;               // tmem base, abort flag, unit ring
+  static constexpr int kTotal = kMisc + 16 + 4 * kUnitRing;
 };
 
 enum DqBar {
   dqQFull = 0, dqQEmpty, dqQtReady, dqKFull0, dqKFull1, dqKFull2, dqKEmpty0, dqKEmpty1, dqKEmpty2,
   dqVFull0, dqVFull1, dqVEmpty0, dqVEmpty1, dqSFull, dqSRead, dqDpFull, dqDsReady, dqDone, dqRead,
-  dqNumBars
+  dqUnitFull0, dqUnitFull1, dqUnitFull2, dqUnitFull3, dqNumBars
 };
 
 // The query-side tiles Q and dO are the stationary A operands of S = Q K^T and dP = dO V^T.
@@ -508,6 +523,7 @@ attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
   auto bar = [&](int i) { return bars + 8u * (uint32_t)i; };
   volatile int* s_tmem = reinterpret_cast<volatile int*>(smem + L::kMisc);
   volatile int* s_abort = s_tmem + 1;
+  volatile int* s_unit = s_tmem + 4;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
@@ -522,6 +538,7 @@ attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
     mbar_init(bar(dqDsReady), kComputeThreads);
     mbar_init(bar(dqDone), 1);
     mbar_init(bar(dqRead), kComputeThreads);
+    for (int i = 0; i < kUnitRing; ++i) mbar_init(bar(dqUnitFull0 + i), 1);
     fence_mbar_init();
     *s_abort = ((sbase & 1023u) != 0) ? 1 : 0;
   }
@@ -541,7 +558,6 @@ attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
   const int G = Hq / Hkv;
   const bool plan_ok = (hdr[PK_HDR_PLAN_T] == T);
   const int n_units = plan_ok ? hdr[PK_HDR_N_ITEMS] * Hq : 0;
-  const int n_cta = gridDim.x, cta = blockIdx.x;
 
   if (warp == kLoadWarp) {
     // =============================== loader ===============================================
@@ -551,8 +567,10 @@ attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
       prefetch_tensormap(&tm_v);
       prefetch_tensormap(&tm_do);
       int gk = 0, uc = 0;
-      for (int r = 0;; ++r, ++uc) {
-        const int u = snake_unit(r, cta, n_cta);
+      for (;; ++uc) {
+        const int u = atomicAdd(&hdr[kHdrDqTicket], 1);
+        s_unit[uc % kUnitRing] = u;
+        mbar_arrive(bar(dqUnitFull0 + uc % kUnitRing));
         if (u >= n_units || *s_abort) break;
         const int4 it = items[order[u / Hq]];
         const int h = u % Hq, g = h / G;
@@ -627,8 +645,9 @@ attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         }
         __syncwarp();
       };
-      for (int r = 0;; ++r, ++uc) {
-        const int u = snake_unit(r, cta, n_cta);
+      for (;; ++uc) {
+        mbar_wait(bar(dqUnitFull0 + uc % kUnitRing), (uc / kUnitRing) & 1, s_abort);
+        const int u = s_unit[uc % kUnitRing];
         if (u >= n_units || *s_abort) break;
         const int4 it = items[order[u / Hq]];
         const int n_kv = (it.w + kBN - 1) / kBN;
@@ -694,9 +713,13 @@ attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
       mbar_arrive(bar(dqQEmpty));
     };
     int gk = 0, uc = 0;
-    if (snake_unit(0, cta, n_cta) < n_units && !*s_abort) copy_q_do(0);
-    for (int r = 0;; ++r, ++uc) {
-      const int u = snake_unit(r, cta, n_cta);
+    auto unit_at = [&](int n) {   // position drawn for this CTA's n-th unit (>= n_units: none)
+      mbar_wait(bar(dqUnitFull0 + n % kUnitRing), (n / kUnitRing) & 1, s_abort);
+      return static_cast<int>(s_unit[n % kUnitRing]);
+    };
+    if (unit_at(0) < n_units && !*s_abort) copy_q_do(0);
+    for (;; ++uc) {
+      const int u = unit_at(uc);
       if (u >= n_units || *s_abort) break;
       const int4 it = items[order[u / Hq]];
       const int h = u % Hq;
@@ -753,7 +776,7 @@ attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
       }
       // The last S and dP of this unit have been consumed, so Q/dO of the NEXT unit can move into
       // tensor memory now; the issuing warp then starts that unit while this one's dQ is written.
-      if (snake_unit(r + 1, cta, n_cta) < n_units && !*s_abort) copy_q_do(uc + 1);
+      if (unit_at(uc + 1) < n_units && !*s_abort) copy_q_do(uc + 1);
       // ---- unit epilogue: dQ rows, scaled (column groups 0 and 1 write half a row each) -----
       mbar_wait(bar(dqDone), uc & 1, s_abort);
       tc_fence_after();
@@ -821,6 +844,10 @@ int launch_ws(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& t
   const float* delta = reinterpret_cast<const float*>(ws + lay.off[PK_WS_DELTA]);
   const float2* table = reinterpret_cast<const float2*>(ws + lay.off[PK_WS_ROPE_TABLE]);
   const int grid = sm_count();
+  // the two unit counters (adjacent header slots) start every call at zero
+  static_assert(kHdrDqTicket == kHdrBwdTicket + 1, "one memset covers both counters");
+  if (cudaMemsetAsync(hdr + kHdrBwdTicket, 0, 2 * sizeof(int32_t), stream) != cudaSuccess)
+    return PK_ERR_CUDA;
   {
     TimedLaunch timed(PK_KERNEL_BWD, stream);
     kern_kv<<<grid, kWsThreads, DkvSmem<D>::kTotal, stream>>>(

@@ -11,8 +11,8 @@
 // Tensor memory: [0,128) S_0 / P_0, [128,256) S_1 / P_1, [256,384) O_0, [384,512) O_1.
 // The commit that announces S_t(j) also covers O_t += P_t V of step j-1 (same pipe, in order), so
 // the softmax warps may rescale O_t in tensor memory as soon as they see S_t(j).
-// Units (forward item x head pair) are assigned statically in snake order over the plan's
-// longest-first list.  Every wait is bounded.
+// Units (forward item x head pair) are drawn from a counter in the plan's order (kFwsUnitRing).
+// Every wait is bounded.
 #include <cuda_bf16.h>
 
 #include "attn_common.cuh"
@@ -31,9 +31,13 @@ constexpr int kFwsLoadWarp = 9;
 constexpr float kLog2eF = 1.4426950408889634f;
 constexpr float kLn2F = 0.6931471805599453f;
 
-__device__ __forceinline__ int snake_unit_f(int r, int cta, int n_cta) {
-  return r * n_cta + ((r & 1) ? (n_cta - 1 - cta) : cta);
-}
+// Units are handed out dynamically: the TMA warp draws the next position of the plan's order
+// from a counter in the workspace header and publishes it to the other roles through a ring of
+// four slots in shared memory (one mbarrier per slot).  The order keeps an example's units
+// together (they share K/V tiles in L2) and drawing from it keeps every CTA busy to the end.
+// No role can fall four units behind the TMA warp: it waits for the previous unit's Q tiles to
+// be released before it loads the next one's.
+constexpr int kFwsUnitRing = 4;
 
 template <int D>
 struct FwsSmem {
@@ -44,13 +48,14 @@ struct FwsSmem {
   static constexpr int kKV0 = 2 * kTileBytes;                // stage s: K then V
   static constexpr int kStageBytes = 2 * kTileBytes;
   static constexpr int kBars = kKV0 + 2 * kStageBytes;
-  static constexpr int kMisc = kBars + 16 * 8;
-  static constexpr int kTotal = kMisc + 16;
+  static constexpr int kMisc = kBars + 24 * 8;               // tmem base, abort flag, unit ring
+  static constexpr int kTotal = kMisc + 16 + 4 * kFwsUnitRing;
 };
 
 enum FwsBar {
   fQFull = 0, fQEmpty, fKvFull0, fKvFull1, fKvEmpty0, fKvEmpty1, fSFull0, fSFull1, fPReady0,
-  fPReady1, fOFull0, fOFull1, fORead0, fORead1, fNumBars
+  fPReady1, fOFull0, fOFull1, fORead0, fORead1, fUnitFull0, fUnitFull1, fUnitFull2, fUnitFull3,
+  fNumBars
 };
 
 template <typename OutT>
@@ -74,6 +79,7 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
   auto bar = [&](int i) { return bars + 8u * (uint32_t)i; };
   volatile int* s_tmem = reinterpret_cast<volatile int*>(smem + L::kMisc);
   volatile int* s_abort = s_tmem + 1;
+  volatile int* s_unit = s_tmem + 4;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
@@ -92,6 +98,7 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
     mbar_init(bar(fOFull1), 1);
     mbar_init(bar(fORead0), 128);
     mbar_init(bar(fORead1), 128);
+    for (int i = 0; i < kFwsUnitRing; ++i) mbar_init(bar(fUnitFull0 + i), 1);
     fence_mbar_init();
     *s_abort = ((sbase & 1023u) != 0) ? 1 : 0;
   }
@@ -109,7 +116,6 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
   const bool plan_ok = (hdr[PK_HDR_PLAN_T] == T);
   if (!plan_ok && blockIdx.x == 0 && tid == 0) set_status(hdr, PK_ERR_NO_PLAN, T);
   const int n_units = plan_ok ? hdr[PK_HDR_N_ITEMS] * pairs : 0;
-  const int n_cta = gridDim.x, cta = blockIdx.x;
 
   if (warp == kFwsLoadWarp) {
     // =============================== loader ===============================================
@@ -118,8 +124,10 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
       prefetch_tensormap(&tm_k);
       prefetch_tensormap(&tm_v);
       int gk = 0, uc = 0;
-      for (int r = 0;; ++r, ++uc) {
-        const int u = snake_unit_f(r, cta, n_cta);
+      for (;; ++uc) {
+        const int u = atomicAdd(&hdr[kHdrFwdTicket], 1);
+        s_unit[uc % kFwsUnitRing] = u;
+        mbar_arrive(bar(fUnitFull0 + uc % kFwsUnitRing));
         if (u >= n_units || *s_abort) break;
         const int4 it = items[order[u / pairs]];
         const int h0 = (u % pairs) * 2, g = h0 / G;
@@ -174,8 +182,9 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         }
         __syncwarp();
       };
-      for (int r = 0;; ++r, ++uc) {
-        const int u = snake_unit_f(r, cta, n_cta);
+      for (;; ++uc) {
+        mbar_wait(bar(fUnitFull0 + uc % kFwsUnitRing), (uc / kFwsUnitRing) & 1, s_abort);
+        const int u = s_unit[uc % kFwsUnitRing];
         if (u >= n_units || *s_abort) break;
         const int4 it = items[order[u / pairs]];
         const int n_kv = (it.w + kBN - 1) / kBN;
@@ -224,8 +233,9 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
     const uint32_t tS = tmem + t * 128 + lane_off;
     const uint32_t tO = tmem + 256 + t * 128 + lane_off;
     int gk = 0, uc = 0;
-    for (int r = 0;; ++r, ++uc) {
-      const int u = snake_unit_f(r, cta, n_cta);
+    for (;; ++uc) {
+      mbar_wait(bar(fUnitFull0 + uc % kFwsUnitRing), (uc / kFwsUnitRing) & 1, s_abort);
+      const int u = s_unit[uc % kFwsUnitRing];
       if (u >= n_units || *s_abort) break;
       const int4 it = items[order[u / pairs]];
       const int h = (u % pairs) * 2 + t;
@@ -326,6 +336,8 @@ int launch_fws(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& 
                            FwsSmem<D>::kTotal) != cudaSuccess)
     return PK_ERR_CUDA;
   int32_t* hdr = reinterpret_cast<int32_t*>(ws + lay.off[PK_WS_HEADER]);
+  if (cudaMemsetAsync(hdr + kHdrFwdTicket, 0, sizeof(int32_t), stream) != cudaSuccess)
+    return PK_ERR_CUDA;
   TimedLaunch timed(PK_KERNEL_FWD, stream);
   kern<<<sm_count(), kFwsThreads, FwsSmem<D>::kTotal, stream>>>(
       tq, tk, tv, reinterpret_cast<const int4*>(ws + lay.off[PK_WS_FWD_ITEMS]),

@@ -17,7 +17,8 @@ constexpr int kHeaderInts = 32;
 
 // header slots beyond the public PK_HDR_* ones
 constexpr int kHdrFwdTicket = 8;
-constexpr int kHdrBwdTicket = 9;
+constexpr int kHdrBwdTicket = 9;    // dK/dV kernel (and the single-kernel backward)
+constexpr int kHdrDqTicket = 10;    // dQ kernel
 
 struct WorkspaceLayout {
   size_t off[PK_WS_NUM_SECTIONS];

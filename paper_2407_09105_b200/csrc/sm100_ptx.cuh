@@ -224,6 +224,22 @@ __device__ __forceinline__ float fast_exp2(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
+// 2^x for x <= 0 without the special-function unit: the exponentials of the attention kernels
+// are bound by that unit (16 results per clock and SM), while the FMA and integer pipes have
+// issue slots to spare, so one exponential in four goes this way.  x is rounded to the nearest
+// integer n by adding 1.5 * 2^23 (n then sits in the low mantissa bits of the sum), 2^(x - n)
+// with x - n in [-0.5, 0.5] is a cubic whose relative error stays below 1.1e-4 (a fraction of
+// the bf16 rounding that follows), and n is added into the exponent field.  No conversion
+// instruction is used: those share the special-function unit's pipe.
+__device__ __forceinline__ float poly_exp2(float x) {
+  x = fmaxf(x, -125.f);                     // keeps the exponent arithmetic in range; 2^-125 is 0 here
+  const float t = x + 12582912.f;           // 1.5 * 2^23
+  const float f = x - (t - 12582912.f);
+  float r = fmaf(f, 0.05500893f, 0.24221095f);
+  r = fmaf(r, f, 0.6932829f);
+  r = fmaf(r, f, 1.0f);
+  return __int_as_float(__float_as_int(r) + (__float_as_int(t) << 23));
+}
 __device__ __forceinline__ uint32_t pack_f16x2(float lo, float hi) {
   uint32_t r;
   asm("cvt.rn.satfinite.f16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
