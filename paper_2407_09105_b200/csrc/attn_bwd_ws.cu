@@ -55,9 +55,6 @@ constexpr float kLog2eWs = 1.4426950408889634f;
 // tiles to be released before it loads the next one's.
 constexpr int kUnitRing = 4;
 
-__device__ __forceinline__ void compute_bar_sync() {
-  asm volatile("bar.sync 1, %0;" ::"n"(kComputeThreads) : "memory");
-}
 
 // =========================================================================================
 // dK / dV kernel
@@ -550,7 +547,7 @@ attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = static_cast<uint32_t>(*s_tmem);
-  // [0,128) S, [128,256) dP (dS as bf16 reuses its first 64 columns), [256,256+D) dQ,
+  // [0,128) S, [128,256) dP (dS as bf16 goes over each thread's own dP columns), [256,256+D) dQ,
   // [384,384+D/2) Q as bf16 pairs, then D/2 columns of dO
   const uint32_t tS = tmem, tdP = tmem + 128, tdQ = tmem + 256, tQ = tmem + 384,
                  tdO = tmem + 384 + D / 2;
@@ -669,9 +666,9 @@ attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
           tc_fence_after();
           if (leader) {
 #pragma unroll
-            for (int kk = 0; kk < kBN / 16; ++kk)   // dQ += dS K   (dS from tensor memory)
-              mma_ts(tdQ, tdP + kk * 8, desc_from_lo(k_lo + ((kk * 2048) >> 4)), kIdescDQ,
-                     (j > 0) | (kk > 0));
+            for (int kk = 0; kk < kBN / 16; ++kk)   // dQ += dS K   (dS of keys 16kk.. : see compute)
+              mma_ts(tdQ, tdP + (kk / (kCW / 16)) * kCW + (kk % (kCW / 16)) * 8,
+                     desc_from_lo(k_lo + ((kk * 2048) >> 4)), kIdescDQ, (j > 0) | (kk > 0));
             mma_commit(bar(dqKEmpty0 + ks));
           }
           __syncwarp();
@@ -764,12 +761,10 @@ attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             dd[c2 * 16 + (e >> 1)] = kRot ? pack_f16x2(d0, d1) : pack_bf16x2(d0, d1);
           }
         }
-        // every thread must have read dP before dS overwrites its columns
-        tc_fence_before();
-        compute_bar_sync();
-        tc_fence_after();
-        if (kCW == 64) tmem_st32(tdP + lane_off + qd * (kCW / 2), dd);
-        else tmem_st16(tdP + lane_off + qd * (kCW / 2), dd);
+        // dS (bf16 pairs, kCW / 2 columns) goes over the first half of this thread's own dP columns:
+        // nobody else reads those, so no block-wide barrier is needed
+        if (kCW == 64) tmem_st32(tdP + lane_off + qd * kCW, dd);
+        else tmem_st16(tdP + lane_off + qd * kCW, dd);
         tmem_wait_st();
         tc_fence_before();
         mbar_arrive(bar(dqDsReady));
