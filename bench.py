@@ -183,6 +183,116 @@ def run_reference(args, w):
     print(json.dumps(line))
 
 
+def run_loss(args):
+    """`--workload loss`: the packed-stream loss (the step after the model), forward + backward
+    over bf16 logits of the first two 8192-token packs of c4 against a 32000-entry vocabulary
+    (Mistral / Llama-2 size).  HBM-bound: the forward reads every logit once, the backward
+    reads it again and writes its gradient.  Prints one JSON line of its own."""
+    from paper_2407_09105_b200 import api
+    from oracle import packed_loss as pl
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
+    w = wl.workload("c4")
+    lens = [x for stream in w.streams[:2] for x in stream]
+    T, V = sum(lens), 32000
+    rng = np.random.default_rng(1234)
+    labels_np = np.concatenate([np.r_[-100, rng.integers(0, V, size=n - 1)] for n in lens]).astype(np.int32)
+    gen = torch.Generator(device="cuda").manual_seed(99)
+    logits = torch.empty((T, V), dtype=torch.bfloat16, device="cuda")
+    for i in range(0, T, 2048):                      # bounded temporaries
+        n = min(2048, T - i)
+        logits[i:i + n] = (torch.randn((n, V), generator=gen, device="cuda") * 2.5).to(torch.bfloat16)
+    labels = torch.tensor(labels_np, device="cuda")
+    dlogits = torch.empty_like(logits)
+    token_loss = torch.empty((T,), device="cuda")
+    lse = torch.empty((T,), device="cuda")
+    result = torch.empty((2,), device="cuda")
+    n_valid = torch.empty((1,), dtype=torch.int32, device="cuda")
+    stream = torch.cuda.current_stream()
+
+    def step():
+        api.pk_packed_loss_fwd(logits, labels, token_loss, lse, result, n_valid, stream=stream)
+        api.pk_packed_loss_bwd(logits, labels, lse, n_valid, 1.0, dlogits, stream=stream)
+
+    kev = {k: [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+               for _ in range(args.steps)] for k in (api.PK_KERNEL_LOSS_FWD, api.PK_KERNEL_LOSS_BWD)}
+    for pairs in kev.values():                       # torch creates the events on first record
+        for a, b in pairs:
+            a.record(stream)
+            b.record(stream)
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(torch.cuda.current_device())
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(args.steps):
+        for k in kev:
+            api.pk_set_timing_events(k, kev[k][i][0], kev[k][i][1])
+        step()
+    e1.record()
+    torch.cuda.synchronize()
+    for k in kev:
+        api.pk_set_timing_events(k, None, None)
+    clocks = sampler.stop()
+    ms = e0.elapsed_time(e1) / args.steps
+    fwd_ms = float(np.mean([a.elapsed_time(b) for a, b in kev[api.PK_KERNEL_LOSS_FWD]]))
+    bwd_ms = float(np.mean([a.elapsed_time(b) for a, b in kev[api.PK_KERNEL_LOSS_BWD]]))
+    peaks = _peaks()
+    fwd_bytes, bwd_bytes = 2.0 * T * V, 4.0 * T * V
+    # end to end: logits from pinned host memory every step, the scalar loss and the gradient back
+    e2e = None
+    if not args.no_e2e:
+        h_logits = torch.empty((T, V), dtype=torch.bfloat16).pin_memory()
+        h_logits.copy_(logits)
+        h_dl = torch.empty((T, V), dtype=torch.bfloat16).pin_memory()
+        h_res = torch.empty((2,)).pin_memory()
+        n_e2e = max(2, min(args.steps, 5))
+        torch.cuda.synchronize()
+        a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a0.record()
+        for _ in range(n_e2e):
+            logits.copy_(h_logits, non_blocking=True)
+            step()
+            h_dl.copy_(dlogits, non_blocking=True)
+            h_res.copy_(result, non_blocking=True)
+        a1.record()
+        torch.cuda.synchronize()
+        e_ms = a0.elapsed_time(a1) / n_e2e
+        e2e = {"value": T / (e_ms * 1e-3), "unit": "tokens/s", "ms_per_step": e_ms,
+               "h2d_bytes_per_step": int(fwd_bytes), "d2h_bytes_per_step": int(fwd_bytes) + 8}
+    cpu = None
+    if not args.no_cpu_baseline:
+        rows = 256                                    # whole leading examples would be too slow
+        x = logits[:rows].float().cpu().numpy().astype(np.float64)
+        t0 = time.perf_counter()
+        pl.loss_fwd(x, labels_np[:rows])
+        pl.loss_bwd(x, labels_np[:rows])
+        dt = time.perf_counter() - t0
+        cpu = {"value": rows / dt, "unit": "tokens/s", "cores": 1, "kind": "oracle",
+               "sample": f"first {rows} rows of the stream, forward + backward in fp64 numpy"}
+    line = {
+        "metric": "packed_loss_fwd_bwd_tokens_per_s", "value": T / (ms * 1e-3), "unit": "tokens/s",
+        "n_gpus": 1, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+        "data": "synthetic",
+        "config": {"workload": "loss: first 2 packs of c4 (16363 tokens) x vocabulary 32000, bf16 logits",
+                   "tokens": T, "vocab": V, "l2": "inputs_exceed_l2"},
+        "clocks": clocks, "e2e": e2e, "gpu_launches": 3 * args.steps,
+        "roofline": {"kernel": "ce_bwd_kernel", "bound": "hbm", "achieved": bwd_bytes / (bwd_ms * 1e-3) / 1e9,
+                     "peak": peaks["hbm_gbs"], "peak_kind": "copy bandwidth, " + peaks["source"],
+                     "unit": "GB/s", "frac": bwd_bytes / (bwd_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                     # 3.9039 B per logit: profiles/loss_kernels_2packs_vocab32000.txt (read + write)
+                     "traffic": 3.9039 * T * V, "ms_per_launch": bwd_ms,
+                     "fwd_kernel": {"achieved": fwd_bytes / (fwd_ms * 1e-3) / 1e9,
+                                    "frac": fwd_bytes / (fwd_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                                    "ms_per_launch": fwd_ms}},
+        "cpu_baseline": cpu,
+    }
+    print(json.dumps(line))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -199,6 +309,9 @@ def main():
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl != "reference" else args.warmup
 
+    if args.workload == "loss":
+        run_loss(args)
+        return
     w = wl.workload(args.workload)
     if args.packs > 0:
         w = wl.Workload(f"{w.name}[:{args.packs}]", w.seed, w.num_q_heads, w.num_kv_heads,

@@ -235,6 +235,33 @@ int pk_pack_next_fit(const int32_t* lengths, int32_t n, int32_t capacity, int32_
                      int32_t* bin_of, int32_t* n_bins);
 
 /*
+ * Loss of the packed stream (the step right after the model).  The collator's labels carry -100
+ * in the first position of every example (Sec. 3.4, worked example in Sec. 3.5); a causal
+ * language model scores row t against the label of row t + 1, so with those labels no example
+ * is asked to predict the start of the next one:
+ *   target[t] = labels[t + 1] for t < T - 1, none for the last row; rows whose target equals
+ *   ignore_index (or is not a vocabulary index) do not count
+ *   loss_t = log(sum_v exp(logits[t][v])) - logits[t][target[t]],  loss = sum_t loss_t / n_valid
+ * pk_packed_loss_fwd   logits [T][row_stride] (PK_BF16 or PK_F32, row_stride >= V elements; rows
+ *                      are read with 16-byte loads when V, row_stride and the base allow it),
+ *                      labels int32 [T].  Writes token_loss float [T] (0 for rows without a
+ *                      target), lse float [T] (natural-log logsumexp, 0 for those rows),
+ *                      result float [2] = {mean, sum}, n_valid int32 [1].  The sum runs in a
+ *                      fixed order: the scalars are bitwise reproducible.  T == 0 gives 0, 0, 0.
+ * pk_packed_loss_bwd   dlogits[t][v] = (exp(logits[t][v] - lse[t]) - [v == target[t]]) * grad_out
+ *                      / n_valid for rows with a target, 0 for the others; same dtype and stride
+ *                      as logits (columns >= V of a padded row are left untouched).  lse and
+ *                      n_valid are the forward's outputs (device pointers: no host round trip).
+ * All pointers are device pointers; the calls allocate nothing.
+ */
+int pk_packed_loss_fwd(const void* logits, int32_t logits_dtype, const int32_t* labels, int32_t T,
+                       int32_t V, int64_t row_stride, int32_t ignore_index, float* token_loss,
+                       float* lse, float* result, int32_t* n_valid, void* stream);
+int pk_packed_loss_bwd(const void* logits, int32_t logits_dtype, const int32_t* labels,
+                       const float* lse, const int32_t* n_valid, float grad_out, int32_t T, int32_t V,
+                       int64_t row_stride, int32_t ignore_index, void* dlogits, void* stream);
+
+/*
  * Self-test of the bounded waits (no counterpart in the paper): one small kernel waits on a
  * barrier that nothing will ever signal, for at most `budget_cycles` SM clocks (1 .. 2e9), then
  * records PK_ERR_TIMEOUT (detail 99) in the status word of `workspace` (>= 128 bytes, its header
@@ -256,7 +283,9 @@ int pk_selftest_bounded_wait(void* workspace, int64_t budget_cycles, void* strea
 #define PK_KERNEL_BWD       3   /* dK/dV kernel (the whole backward when RoPE is fused) */
 #define PK_KERNEL_DQ_FINISH 4
 #define PK_KERNEL_BWD_DQ    5   /* dQ kernel */
-#define PK_NUM_KERNELS      6
+#define PK_KERNEL_LOSS_FWD  6   /* row pass of pk_packed_loss_fwd */
+#define PK_KERNEL_LOSS_BWD  7
+#define PK_NUM_KERNELS      8
 int pk_set_timing_events(int32_t which, void* start, void* stop);
 
 #ifdef __cplusplus

@@ -53,6 +53,10 @@ _SIGNATURES = {
     "pk_collate_padding_free": (ctypes.c_int, [_vp, _vp, _i32, _i32, _vp, _vp, _vp, _i32, _vp]),
     "pk_pack_first_fit_decreasing": (ctypes.c_int, [_vp, _i32, _i32, _vp, ctypes.POINTER(_i32)]),
     "pk_pack_next_fit": (ctypes.c_int, [_vp, _i32, _i32, _i32, _vp, ctypes.POINTER(_i32)]),
+    "pk_packed_loss_fwd": (ctypes.c_int, [_vp, _i32, _vp, _i32, _i32, ctypes.c_int64, _i32, _vp, _vp,
+                                          _vp, _vp, _vp]),
+    "pk_packed_loss_bwd": (ctypes.c_int, [_vp, _i32, _vp, _vp, _vp, ctypes.c_float, _i32, _i32,
+                                          ctypes.c_int64, _i32, _vp, _vp]),
     "pk_selftest_bounded_wait": (ctypes.c_int, [_vp, ctypes.c_int64, _vp]),
     "pk_seqlens_from_posids_noalloc": (ctypes.c_int, [_vp, _i32, _vp, _vp, _vp, _vp]),
 }
@@ -201,7 +205,8 @@ def pk_status_read(workspace: torch.Tensor, stream=None) -> Tuple[int, int]:
     return code.value, detail.value
 
 
-PK_KERNEL_PLAN, PK_KERNEL_FWD, PK_KERNEL_DELTA, PK_KERNEL_BWD, PK_KERNEL_DQ_FINISH, PK_KERNEL_BWD_DQ = range(6)
+(PK_KERNEL_PLAN, PK_KERNEL_FWD, PK_KERNEL_DELTA, PK_KERNEL_BWD, PK_KERNEL_DQ_FINISH, PK_KERNEL_BWD_DQ,
+ PK_KERNEL_LOSS_FWD, PK_KERNEL_LOSS_BWD) = range(8)
 
 
 def pk_set_timing_events(which: int, start: Optional[torch.cuda.Event],
@@ -227,6 +232,42 @@ def pk_collate_padding_free(input_ids: torch.Tensor, lengths: torch.Tensor,
            lib().pk_collate_padding_free(_ptr(input_ids), _ptr(lengths), lengths.numel(),
                                          position_ids.numel(), _ptr(position_ids), _ptr(labels),
                                          _ptr(cu_seqlens), ignore_index, _stream(stream)))
+
+
+def _logits_dtype(t: torch.Tensor) -> int:
+    if t.dtype == torch.bfloat16:
+        return PK_BF16
+    if t.dtype == torch.float32:
+        return PK_F32
+    raise ValueError("logits must be bfloat16 or float32")
+
+
+def pk_packed_loss_fwd(logits: torch.Tensor, labels: torch.Tensor, token_loss: torch.Tensor,
+                       lse: torch.Tensor, result: torch.Tensor, n_valid: torch.Tensor,
+                       ignore_index: int = -100, stream=None) -> None:
+    """logits [T, V] (rows may be padded: stride(0) >= V, stride(1) == 1)."""
+    T, V = logits.shape
+    if logits.stride(1) != 1 and T > 0:
+        raise ValueError("logits rows must be contiguous")
+    stride = logits.stride(0) if T > 1 else V
+    _check("pk_packed_loss_fwd",
+           lib().pk_packed_loss_fwd(logits.data_ptr(), _logits_dtype(logits), _ptr(labels), T, V,
+                                    stride, ignore_index, _ptr(token_loss), _ptr(lse),
+                                    _ptr(result), _ptr(n_valid), _stream(stream)))
+
+
+def pk_packed_loss_bwd(logits: torch.Tensor, labels: torch.Tensor, lse: torch.Tensor,
+                       n_valid: torch.Tensor, grad_out: float, dlogits: torch.Tensor,
+                       ignore_index: int = -100, stream=None) -> None:
+    T, V = logits.shape
+    if dlogits.shape != logits.shape or dlogits.dtype != logits.dtype or \
+            dlogits.stride() != logits.stride():
+        raise ValueError("dlogits must match logits in shape, dtype and strides")
+    stride = logits.stride(0) if T > 1 else V
+    _check("pk_packed_loss_bwd",
+           lib().pk_packed_loss_bwd(logits.data_ptr(), _logits_dtype(logits), _ptr(labels),
+                                    _ptr(lse), _ptr(n_valid), float(grad_out), T, V, stride,
+                                    ignore_index, dlogits.data_ptr(), _stream(stream)))
 
 
 def _pack(fn_name, lengths, capacity, *extra):
