@@ -113,7 +113,7 @@ def _launches_per_call(theta, Hq, Hkv, D):
     pairs = (Hq // Hkv) % 2 == 0
     if D == 128:                      # rotated fp16 copies of q and k
         fwd = 4 if pairs else 3       # plan, rotate q, rotate k, forward | plan, table, forward
-        return fwd + 6                # table, delta, rotate q, rotate k, dK/dV, dQ
+        return fwd + (4 if pairs else 6)   # table, delta, dK/dV, dQ (+ rotate q, k if the forward made none)
     return 3 + 4                      # in-tile: plan, table, forward | table, delta, backward, dQ finish
 
 
@@ -362,7 +362,7 @@ def main():
                 api.pk_attn_fwd(q_, k_, v_, pos_, scale, theta, out_, lse_, ws,
                                 reuse_plan=False, stream=stream)
                 api.pk_attn_bwd(do_, q_, k_, v_, out_, lse_, pos_, scale, theta,
-                                dq_, dk_, dv_, ws, reuse_plan=True, stream=stream)
+                                dq_, dk_, dv_, ws, reuse_plan=True, reuse_rotated=True, stream=stream)
         calls_per_step = len(pieces)
     else:
         ws = api.alloc_workspace(T, Hq, Hkv, D)
@@ -371,7 +371,7 @@ def main():
             api.pk_attn_fwd(st.q, st.k, st.v, st.position_ids, scale, theta, out, lse, ws,
                             reuse_plan=False, stream=stream)
             api.pk_attn_bwd(st.dout, st.q, st.k, st.v, out, lse, st.position_ids, scale, theta,
-                            dq, dk, dv, ws, reuse_plan=True, stream=stream)
+                            dq, dk, dv, ws, reuse_plan=True, reuse_rotated=True, stream=stream)
         calls_per_step = 1
 
     def barrier():

@@ -127,9 +127,16 @@ int pk_rope_apply(void* x, const int32_t* position_ids, int32_t T, int32_t H, in
  *                 (q', k'); <= 0: q and k are used as given
  *   out           [T, Hq, D], element type out_dtype (PK_BF16 or PK_F32)
  *   lse           fp32 [Hq, T]
- *   reuse_plan    0: run the planning step of pk_seqlens_from_posids first (same stream);
- *                 1: use the plan already in `workspace` (must be for these position_ids)
+ *   reuse_plan    bit mask.  0: run the planning step of pk_seqlens_from_posids first (same
+ *                 stream); PK_REUSE_PLAN: use the plan already in `workspace` (must be for
+ *                 these position_ids).  pk_attn_bwd also takes PK_REUSE_ROTATED: with
+ *                 rope_theta > 0 the forward leaves rotated copies of q and k in the workspace
+ *                 (default RoPE mode, D = 128, Hq/Hkv even); the flag says that they are
+ *                 still there (same q, k, position_ids, rope_theta; workspace untouched since
+ *                 the forward), so the backward does not make them again.
  */
+#define PK_REUSE_PLAN     1
+#define PK_REUSE_ROTATED  2
 int pk_attn_fwd(const void* q, const void* k, const void* v, const int32_t* position_ids,
                 int32_t T, int32_t Hq, int32_t Hkv, int32_t D,
                 float softmax_scale, float rope_theta,

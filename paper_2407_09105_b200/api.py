@@ -25,6 +25,7 @@ PK_NOALLOC_MAX_TOKENS = 32768
 
 PK_BF16 = 0
 PK_F32 = 1
+PK_REUSE_PLAN, PK_REUSE_ROTATED = 1, 2
 
 PK_WS_HEADER, PK_WS_FWD_ITEMS, PK_WS_BWD_ITEMS, PK_WS_FWD_ORDER, PK_WS_BWD_ORDER = range(5)
 PK_WS_DELTA, PK_WS_DQ_ACC, PK_WS_ROPE_TABLE = 5, 6, 7
@@ -185,7 +186,9 @@ def pk_attn_fwd(q, k, v, position_ids, softmax_scale: float, rope_theta: float,
 
 def pk_attn_bwd(dout, q, k, v, out, lse, position_ids, softmax_scale: float, rope_theta: float,
                 dq: torch.Tensor, dk: torch.Tensor, dv: torch.Tensor, workspace: torch.Tensor,
-                reuse_plan: bool = True, stream=None) -> None:
+                reuse_plan: bool = True, reuse_rotated: bool = False, stream=None) -> None:
+    """``reuse_rotated``: the rotated q / k copies the forward left in ``workspace`` are still
+    valid (same q, k, position_ids, rope_theta; workspace untouched since)."""
     T, Hq, D = q.shape
     Hkv = k.shape[1]
     if not (dq.dtype == dk.dtype == dv.dtype):
@@ -194,7 +197,9 @@ def pk_attn_bwd(dout, q, k, v, out, lse, position_ids, softmax_scale: float, rop
            lib().pk_attn_bwd(_ptr(dout), _ptr(q), _ptr(k), _ptr(v), _ptr(out), _dtype_code(out),
                              _ptr(lse), _ptr(position_ids), T, Hq, Hkv, D, softmax_scale,
                              rope_theta, _ptr(dq), _ptr(dk), _ptr(dv), _dtype_code(dq),
-                             int(reuse_plan), _ptr(workspace), workspace.numel(), _stream(stream)))
+                             (PK_REUSE_PLAN if reuse_plan else 0) |
+                             (PK_REUSE_ROTATED if reuse_rotated else 0),
+                             _ptr(workspace), workspace.numel(), _stream(stream)))
 
 
 def pk_status_read(workspace: torch.Tensor, stream=None) -> Tuple[int, int]:

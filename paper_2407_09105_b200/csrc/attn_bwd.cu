@@ -506,7 +506,7 @@ extern "C" int pk_attn_bwd(const void* dout, const void* q, const void* k, const
 
   char* ws = static_cast<char*>(workspace);
   int rc;
-  if (!reuse_plan) {
+  if (!(reuse_plan & PK_REUSE_PLAN)) {
     rc = plan_launch(position_ids, T, nullptr, nullptr, nullptr, workspace, lay, stream);
     if (rc != PK_OK) return rc;
   }
@@ -550,10 +550,15 @@ extern "C" int pk_attn_bwd(const void* dout, const void* q, const void* k, const
     // rotated fp16 copies of q and k in the dQ accumulator section (not needed otherwise here)
     char* qr = ws + lay.off[PK_WS_DQ_ACC];
     char* kr = qr + align_up((size_t)T * Hq * D * 2, 256);
-    rc = rope_rotate_f16_launch(q, position_ids, T, Hq, D, rope_theta, qr, stream);
-    if (rc != PK_OK) return rc;
-    rc = rope_rotate_f16_launch(k, position_ids, T, Hkv, D, rope_theta, kr, stream);
-    if (rc != PK_OK) return rc;
+    // PK_REUSE_ROTATED: the forward left exactly these copies there (it makes them when the
+    // query heads of a kv head come in pairs) and the caller vouches that nothing touched them
+    const bool have_copies = (reuse_plan & PK_REUSE_ROTATED) != 0 && (Hq / Hkv) % 2 == 0;
+    if (!have_copies) {
+      rc = rope_rotate_f16_launch(q, position_ids, T, Hq, D, rope_theta, qr, stream);
+      if (rc != PK_OK) return rc;
+      rc = rope_rotate_f16_launch(k, position_ids, T, Hkv, D, rope_theta, kr, stream);
+      if (rc != PK_OK) return rc;
+    }
     CUtensorMap tqr, tkr;
     if (!make_tile_map_bf16(&tqr, qr, T, Hq * D) || !make_tile_map_bf16(&tkr, kr, T, Hkv * D))
       return PK_ERR_CUDA;

@@ -352,7 +352,7 @@ extern "C" int pk_attn_fwd(const void* q, const void* k, const void* v,
     return PK_ERR_INVALID_ARG;
 
   char* ws = static_cast<char*>(workspace);
-  if (!reuse_plan) {
+  if (!(reuse_plan & PK_REUSE_PLAN)) {
     int rc = plan_launch(position_ids, T, nullptr, nullptr, nullptr, workspace, lay, stream);
     if (rc != PK_OK) return rc;
   }

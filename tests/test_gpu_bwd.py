@@ -100,3 +100,24 @@ def test_fused_rope_equals_unfused_composition():
     pos = st.position_ids.cpu().numpy()
     assert max_abs(f64(dq), orc.rope(f64(dq2), pos, theta, inverse=True)) <= 2e-2
     assert max_abs(f64(dk), orc.rope(f64(dk2), pos, theta, inverse=True)) <= 2e-2
+
+
+def test_backward_reusing_the_forwards_rotated_copies_is_bitwise_the_same():
+    import numpy as np
+    from paper_2407_09105_b200 import api, workloads as wl
+    lens = [300, 5, 200, 131]
+    w = wl.Workload("t", 11, 8, 2, 128, 1e4, [lens], "test")
+    st = wl.stream_tensors(w, lens, 0, device="cuda")
+    T, Hq, D = st.q.shape
+    ws = api.alloc_workspace(T, Hq, 2, D)
+    out = torch.empty_like(st.q)
+    lse = torch.empty((Hq, T), dtype=torch.float32, device="cuda")
+    res = []
+    for reuse in (False, True):
+        api.pk_attn_fwd(st.q, st.k, st.v, st.position_ids, w.softmax_scale, w.rope_theta, out, lse, ws)
+        dq, dk, dv = torch.empty_like(st.q), torch.empty_like(st.k), torch.empty_like(st.v)
+        api.pk_attn_bwd(st.dout, st.q, st.k, st.v, out, lse, st.position_ids, w.softmax_scale,
+                        w.rope_theta, dq, dk, dv, ws, reuse_plan=True, reuse_rotated=reuse)
+        torch.cuda.synchronize()
+        res.append([x.float().cpu().numpy().tobytes() for x in (dq, dk, dv)])
+    assert res[0] == res[1]
