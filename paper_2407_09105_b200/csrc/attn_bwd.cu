@@ -550,9 +550,9 @@ extern "C" int pk_attn_bwd(const void* dout, const void* q, const void* k, const
     // rotated fp16 copies of q and k in the dQ accumulator section (not needed otherwise here)
     char* qr = ws + lay.off[PK_WS_DQ_ACC];
     char* kr = qr + align_up((size_t)T * Hq * D * 2, 256);
-    // PK_REUSE_ROTATED: the forward left exactly these copies there (it makes them when the
-    // query heads of a kv head come in pairs) and the caller vouches that nothing touched them
-    const bool have_copies = (reuse_plan & PK_REUSE_ROTATED) != 0 && (Hq / Hkv) % 2 == 0;
+    // PK_REUSE_ROTATED: the forward left exactly these copies there and the caller vouches that
+    // nothing touched them
+    const bool have_copies = (reuse_plan & PK_REUSE_ROTATED) != 0;
     if (!have_copies) {
       rc = rope_rotate_f16_launch(q, position_ids, T, Hq, D, rope_theta, qr, stream);
       if (rc != PK_OK) return rc;

@@ -357,8 +357,7 @@ extern "C" int pk_attn_fwd(const void* q, const void* k, const void* v,
     if (rc != PK_OK) return rc;
   }
   const bool use_rope = rope_theta > 0.f;
-  const bool ws_shape = (Hq / Hkv) % 2 == 0;
-  if (use_rope && g_rope_mode == PK_ROPE_ROTATED_COPIES && D == 128 && ws_shape) {
+  if (use_rope && g_rope_mode == PK_ROPE_ROTATED_COPIES && D == 128) {
     // rotated fp16 copies of q and k in the (otherwise unused) dQ accumulator section
     char* qr = ws + lay.off[PK_WS_DQ_ACC];
     char* kr = qr + align_up((size_t)T * Hq * D * 2, 256);
@@ -383,7 +382,7 @@ extern "C" int pk_attn_fwd(const void* q, const void* k, const void* v,
       !make_tile_map_bf16(&tv, v, T, Hkv * D))
     return PK_ERR_CUDA;
 
-  if (!use_rope && ws_shape)   // two query heads of a kv head per CTA, warp-specialised
+  if (!use_rope)   // two tiles per CTA (two heads of a kv head, or two query blocks), warp-specialised
     return launch_fwd_ws(tq, tk, tv, ws, lay, out, lse, T, Hq, Hkv, D, out_dtype, softmax_scale,
                          false, stream);
 #define PK_FWD(DD, RR, TT) \

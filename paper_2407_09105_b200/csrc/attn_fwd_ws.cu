@@ -11,7 +11,8 @@
 // Tensor memory: [0,128) S_0 / P_0, [128,256) S_1 / P_1, [256,384) O_0, [384,512) O_1.
 // The commit that announces S_t(j) also covers O_t += P_t V of step j-1 (same pipe, in order), so
 // the softmax warps may rescale O_t in tensor memory as soon as they see S_t(j).
-// Units (forward item x head pair) are drawn from a counter in the plan's order (kFwsUnitRing).
+// Units (forward item x head pair, or pair of query blocks x head: see FwdUnit) are drawn from a
+// counter in the plan's order (kFwsUnitRing).
 // Every wait is bounded.
 #include <cuda_bf16.h>
 
@@ -66,12 +67,61 @@ __device__ __forceinline__ void store_out32(OutT* dst, const uint32_t* r, float 
   store_chunk32<OutT>(dst, y);
 }
 
+// What the two tiles of a unit are.  With an even number of query heads per kv head they are two
+// query heads of one kv head over the same query block.  Otherwise (multi-head attention, odd
+// group sizes) they are two consecutive query blocks b-1 and b of one example and one head, which
+// also share every K/V tile: the unit runs the b+1 key steps of block b, and block b-1 sees its
+// diagonal one step earlier and nothing in the last step.  Blocks are paired from the end of the
+// example, so a block is left over only when the count is odd, and then it is block 0 (one key
+// step), which runs with a copy of itself as tile 0 whose results are not stored.
+struct FwdUnit {
+  int h[2], q_start[2], q_len[2], diag[2];   // per tile: head, rows, rows to store, diagonal step
+  int g, kv_start, n_kv;
+};
+__device__ __forceinline__ FwdUnit decode_fwd_unit(int u, const int4* __restrict__ items,
+                                                   const int32_t* __restrict__ order, int Hq,
+                                                   int G, bool pair_blocks) {
+  FwdUnit w;
+  if (!pair_blocks) {
+    const int pairs = Hq / 2;
+    const int4 it = items[order[u / pairs]];
+    const int h0 = (u % pairs) * 2;
+    w.n_kv = (it.w + kBN - 1) / kBN;
+    w.kv_start = it.z;
+    w.g = h0 / G;
+#pragma unroll
+    for (int t = 0; t < 2; ++t) {
+      w.h[t] = h0 + t; w.q_start[t] = it.x; w.q_len[t] = it.y; w.diag[t] = w.n_kv - 1;
+    }
+  } else {
+    const int4 it = items[order[u / Hq]];
+    const int h = u % Hq;
+    const int b = (it.x - it.z) / kBM;          // block index inside the example
+    w.n_kv = b + 1;
+    w.kv_start = it.z;
+    w.g = h / G;
+    w.h[0] = w.h[1] = h;
+    w.q_start[1] = it.x; w.q_len[1] = it.y; w.diag[1] = b;
+    if (b >= 1) { w.q_start[0] = it.x - kBM; w.q_len[0] = kBM; w.diag[0] = b - 1; }
+    else        { w.q_start[0] = it.x;       w.q_len[0] = 0;   w.diag[0] = 0; }
+  }
+  return w;
+}
+// block-pair mode: item n leads a unit when an even number of blocks follows it in its example
+// (the backward item of the same index holds the rows from this block to the example's end)
+__device__ __forceinline__ bool leads_block_pair(int u, const int4* __restrict__ bwd_items,
+                                                 const int32_t* __restrict__ order, int Hq) {
+  const int4 bi = bwd_items[order[u / Hq]];
+  return (((bi.w + kBM - 1) / kBM - 1) & 1) == 0;
+}
+
 template <int D, bool kRot, typename OutT>
 __global__ void __launch_bounds__(kFwsThreads, 1)
 attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                    const __grid_constant__ CUtensorMap tm_v, const int4* __restrict__ items,
-                   const int32_t* __restrict__ order, int32_t* hdr, OutT* __restrict__ out,
-                   float* __restrict__ lse, int T, int Hq, int Hkv, float scale_log2) {
+                   const int4* __restrict__ bwd_items, const int32_t* __restrict__ order,
+                   int32_t* hdr, OutT* __restrict__ out, float* __restrict__ lse, int T, int Hq,
+                   int Hkv, float scale_log2) {
   using L = FwsSmem<D>;
   extern __shared__ __align__(1024) uint8_t smem[];
   const uint32_t sbase = smem_u32(smem);
@@ -112,10 +162,10 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
   const uint32_t tmem = static_cast<uint32_t>(*s_tmem);
 
   const int G = Hq / Hkv;
-  const int pairs = Hq / 2;
+  const bool pair_blocks = (G % 2) != 0;
   const bool plan_ok = (hdr[PK_HDR_PLAN_T] == T);
   if (!plan_ok && blockIdx.x == 0 && tid == 0) set_status(hdr, PK_ERR_NO_PLAN, T);
-  const int n_units = plan_ok ? hdr[PK_HDR_N_ITEMS] * pairs : 0;
+  const int n_units = plan_ok ? hdr[PK_HDR_N_ITEMS] * (pair_blocks ? Hq : Hq / 2) : 0;
 
   if (warp == kFwsLoadWarp) {
     // =============================== loader ===============================================
@@ -125,14 +175,15 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
       prefetch_tensormap(&tm_v);
       int gk = 0, uc = 0;
       for (;; ++uc) {
-        const int u = atomicAdd(&hdr[kHdrFwdTicket], 1);
+        int u;
+        do {   // in block-pair mode only the leading block of a pair becomes a unit
+          u = atomicAdd(&hdr[kHdrFwdTicket], 1);
+        } while (u < n_units && pair_blocks && !leads_block_pair(u, bwd_items, order, Hq));
         s_unit[uc % kFwsUnitRing] = u;
         mbar_arrive(bar(fUnitFull0 + uc % kFwsUnitRing));
         if (u >= n_units || *s_abort) break;
-        const int4 it = items[order[u / pairs]];
-        const int h0 = (u % pairs) * 2, g = h0 / G;
-        const int q_start = it.x, kv_start = it.z, kv_len = it.w;
-        const int n_kv = (kv_len + kBN - 1) / kBN;
+        const FwdUnit w = decode_fwd_unit(u, items, order, Hq, G, pair_blocks);
+        const int g = w.g, kv_start = w.kv_start, n_kv = w.n_kv;
         mbar_wait(bar(fQEmpty), (uc & 1) ^ 1, s_abort);
         mbar_expect_tx(bar(fQFull), 2 * L::kTileBytes);
 #pragma unroll
@@ -140,7 +191,7 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
 #pragma unroll
           for (int b = 0; b < L::kBoxes; ++b)
             tma_load_2d(sbase + L::kQ0 + t * L::kTileBytes + b * L::kBoxBytes, &tm_q,
-                        (h0 + t) * D + b * 64, q_start, bar(fQFull));
+                        w.h[t] * D + b * 64, w.q_start[t], bar(fQFull));
         for (int j = 0; j < n_kv; ++j, ++gk) {
           const int st = gk & 1;
           const uint32_t sK = sbase + L::kKV0 + st * L::kStageBytes, sV = sK + L::kTileBytes;
@@ -186,8 +237,7 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         mbar_wait(bar(fUnitFull0 + uc % kFwsUnitRing), (uc / kFwsUnitRing) & 1, s_abort);
         const int u = s_unit[uc % kFwsUnitRing];
         if (u >= n_units || *s_abort) break;
-        const int4 it = items[order[u / pairs]];
-        const int n_kv = (it.w + kBN - 1) / kBN;
+        const int n_kv = decode_fwd_unit(u, items, order, Hq, G, pair_blocks).n_kv;
         mbar_wait(bar(fQFull), uc & 1, s_abort);
         mbar_wait(bar(fKvFull0 + (gk & 1)), (gk >> 1) & 1, s_abort);
         tc_fence_after();
@@ -237,10 +287,9 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
       mbar_wait(bar(fUnitFull0 + uc % kFwsUnitRing), (uc / kFwsUnitRing) & 1, s_abort);
       const int u = s_unit[uc % kFwsUnitRing];
       if (u >= n_units || *s_abort) break;
-      const int4 it = items[order[u / pairs]];
-      const int h = (u % pairs) * 2 + t;
-      const int q_start = it.x, q_len = it.y, kv_len = it.w;
-      const int n_kv = (kv_len + kBN - 1) / kBN;
+      const FwdUnit w = decode_fwd_unit(u, items, order, Hq, G, pair_blocks);
+      const int h = w.h[t], q_start = w.q_start[t], q_len = w.q_len[t], diag = w.diag[t];
+      const int n_kv = w.n_kv;
       float m_run = -INFINITY, l_run = 0.f;
       for (int j = 0; j < n_kv; ++j, ++gk) {
         mbar_wait(bar(fSFull0 + t), gk & 1, s_abort);
@@ -249,10 +298,12 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
 #pragma unroll
         for (int c = 0; c < 4; ++c) tmem_ld32(tS + c * 32, s + c * 32);
         tmem_wait_ld();
-        if (j == n_kv - 1) {   // diagonal tile: keys after the query row are masked
+        if (j >= diag) {       // diagonal tile: keys after the query row are masked; a tile past
+                               // the diagonal (block-pair mode, tile 0, last step) entirely
+          const int first_masked = (j == diag) ? row + 1 : 0;
 #pragma unroll
           for (int c = 0; c < 128; ++c)
-            if (c > row) s[c] = 0xff800000u;   // -inf
+            if (c >= first_masked) s[c] = 0xff800000u;   // -inf
         }
         float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};   // independent chains
 #pragma unroll
@@ -341,6 +392,7 @@ int launch_fws(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& 
   TimedLaunch timed(PK_KERNEL_FWD, stream);
   kern<<<sm_count(), kFwsThreads, FwsSmem<D>::kTotal, stream>>>(
       tq, tk, tv, reinterpret_cast<const int4*>(ws + lay.off[PK_WS_FWD_ITEMS]),
+      reinterpret_cast<const int4*>(ws + lay.off[PK_WS_BWD_ITEMS]),
       reinterpret_cast<const int32_t*>(ws + lay.off[PK_WS_FWD_ORDER]), hdr,
       static_cast<OutT*>(out), lse, T, Hq, Hkv, scale * kLog2eF);
   return launch_status();

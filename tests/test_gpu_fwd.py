@@ -43,6 +43,16 @@ def test_tile_edges(D, lens):
     _case(lens, 2, 2, D, 0.0, seed=3)
 
 
+@pytest.mark.parametrize("Hq,Hkv", [(2, 2), (3, 1), (6, 2)])
+def test_odd_group_sizes_pair_query_blocks(Hq, Hkv):
+    # with an odd number of query heads per kv head a unit is two consecutive query blocks of one
+    # example: block counts 1 .. 7 cover the left-over block 0, the masked last step of the
+    # shorter block, and ragged last blocks
+    _case([1, 128, 129, 256, 257, 384, 385, 641, 896, 100], Hq, Hkv, 128, 0.0, seed=21)
+    _case([513, 2, 300], Hq, Hkv, 64, 0.0, seed=22, out_dtype=torch.bfloat16)
+    _case([385, 130], Hq, Hkv, 128, 1e4, seed=23)         # rotated copies
+
+
 @pytest.mark.parametrize("D", [64, 128])
 def test_gqa(D):
     _case([200, 77, 400], 8, 2, D, 0.0, seed=4)
@@ -54,7 +64,7 @@ def test_fused_rope(D, theta, mode):
     api.pk_set_rope_mode(mode)
     try:
         _case([150, 260, 3, 129], 4, 2, D, theta, seed=5)
-        _case([300, 40], 4, 4, D, theta, seed=15)          # MHA: the forward stays in-tile
+        _case([300, 40], 4, 4, D, theta, seed=15)          # MHA: block pairs share K/V tiles
     finally:
         api.pk_set_rope_mode(api.PK_ROPE_ROTATED_COPIES)
 
