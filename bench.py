@@ -110,9 +110,8 @@ def _launches_per_call(theta, Hq, Hkv, D):
     """Kernels of this library per forward+backward pair (default RoPE mode)."""
     if theta <= 0:
         return 5                      # plan, forward, delta, dK/dV, dQ
-    if D == 128:                      # rotated fp16 copies of q and k, made once by the forward
-        return 4 + 4                  # plan, rotate q, rotate k, forward | table, delta, dK/dV, dQ
-    return 3 + 4                      # in-tile: plan, table, forward | table, delta, backward, dQ finish
+    # rotated fp16 copies of q and k, made once by the forward:
+    return 4 + 4                      # plan, rotate q, rotate k, forward | table, delta, dK/dV, dQ
 
 
 def _oracle_sample(w: wl.Workload):

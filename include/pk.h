@@ -131,7 +131,7 @@ int pk_rope_apply(void* x, const int32_t* position_ids, int32_t T, int32_t H, in
  *                 stream); PK_REUSE_PLAN: use the plan already in `workspace` (must be for
  *                 these position_ids).  pk_attn_bwd also takes PK_REUSE_ROTATED: with
  *                 rope_theta > 0 the forward leaves rotated copies of q and k in the workspace
- *                 (default RoPE mode, D = 128, Hq/Hkv even); the flag says that they are
+ *                 (default RoPE mode); the flag says that they are
  *                 still there (same q, k, position_ids, rope_theta; workspace untouched since
  *                 the forward), so the backward does not make them again.
  */

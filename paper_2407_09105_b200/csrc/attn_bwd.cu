@@ -511,7 +511,7 @@ extern "C" int pk_attn_bwd(const void* dout, const void* q, const void* k, const
     if (rc != PK_OK) return rc;
   }
   const bool use_rope = rope_theta > 0.f;
-  const bool rotated_copies = use_rope && g_rope_mode == PK_ROPE_ROTATED_COPIES && D == 128;
+  const bool rotated_copies = use_rope && g_rope_mode == PK_ROPE_ROTATED_COPIES;
   float* table = reinterpret_cast<float*>(ws + lay.off[PK_WS_ROPE_TABLE]);
   if (use_rope) {
     rc = rope_table_launch(position_ids, T, D, rope_theta, table, stream);

@@ -429,13 +429,13 @@ attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         const float mul = is_dv ? 1.f : scale;
         if (kRot && !is_dv) {
           // dK was formed against the rotated k: rotate back by -angle, pairs (i, i + D/2)
-          static_assert(!kRot || (D == 128 && kEpiCols == 128), "rotated path is built for D = 128");
+          static_assert(!kRot || kEpiCols == D, "one thread holds both halves of a dK row");
 #pragma unroll
-          for (int c = 0; c < 2; ++c) {
+          for (int c = 0; c < D / 64; ++c) {
             uint32_t x1[32], x2[32];
             float y1[32], y2[32];
             tmem_ld32(src + c * 32, x1);
-            tmem_ld32(src + 64 + c * 32, x2);
+            tmem_ld32(src + D / 2 + c * 32, x2);
             tmem_wait_ld();
             if (live) {
               const float2* cs = rope_table + (size_t)tok * (D / 2) + c * 32;
@@ -447,7 +447,7 @@ attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 y2[e] = b * t.x - a * t.y;
               }
               store_chunk32<GradT>(dst + c * 32, y1);
-              store_chunk32<GradT>(dst + 64 + c * 32, y2);
+              store_chunk32<GradT>(dst + D / 2 + c * 32, y2);
             }
           }
         } else {
@@ -778,15 +778,19 @@ attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
       if (qd < 2) {
         const bool live = (row < q_len) && (*s_abort == 0);
         if (kRot) {
-          // rotate back by -angle: this thread owns pairs i in [32*qd, +32) and i + 64
-          static_assert(!kRot || D == 128, "rotated path is built for D = 128");
+          // rotate back by -angle: this thread owns pairs i in [32*qd, +32) and i + D/2 (with
+          // D = 64 there are only 32 pairs: column group 0 takes them all)
+          static_assert(!kRot || D == 128 || D == 64, "rotated path is built for D = 64 and 128");
           GradT* dst = dq + ((size_t)tok * Hq + h) * D + qd * 32;
           uint32_t x1[32], x2[32];
           float y1[32], y2[32];
-          tmem_ld32(tdQ + lane_off + qd * 32, x1);
-          tmem_ld32(tdQ + lane_off + 64 + qd * 32, x2);
+          const bool mine = qd * 32 < D / 2;
+          if (mine) {
+            tmem_ld32(tdQ + lane_off + qd * 32, x1);
+            tmem_ld32(tdQ + lane_off + D / 2 + qd * 32, x2);
+          }
           tmem_wait_ld();
-          if (live) {
+          if (live && mine) {
             const float2* cs = rope_table + (size_t)tok * (D / 2) + qd * 32;
 #pragma unroll
             for (int e = 0; e < 32; ++e) {
@@ -796,7 +800,7 @@ attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
               y2[e] = b * t.x - a * t.y;
             }
             store_chunk32<GradT>(dst, y1);
-            store_chunk32<GradT>(dst + 64, y2);
+            store_chunk32<GradT>(dst + D / 2, y2);
           }
         } else {
           GradT* dst = dq + ((size_t)tok * Hq + h) * D + qd * (D / 2);
@@ -877,6 +881,9 @@ int launch_bwd_ws(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMa
     } else {
       if (grad_dtype == PK_BF16) PK_BWS(128, false, __nv_bfloat16); else PK_BWS(128, false, float);
     }
+  }
+  if (rotated) {
+    if (grad_dtype == PK_BF16) PK_BWS(64, true, __nv_bfloat16); else PK_BWS(64, true, float);
   }
   if (grad_dtype == PK_BF16) PK_BWS(64, false, __nv_bfloat16);
   PK_BWS(64, false, float);

@@ -357,7 +357,7 @@ extern "C" int pk_attn_fwd(const void* q, const void* k, const void* v,
     if (rc != PK_OK) return rc;
   }
   const bool use_rope = rope_theta > 0.f;
-  if (use_rope && g_rope_mode == PK_ROPE_ROTATED_COPIES && D == 128) {
+  if (use_rope && g_rope_mode == PK_ROPE_ROTATED_COPIES) {
     // rotated fp16 copies of q and k in the (otherwise unused) dQ accumulator section
     char* qr = ws + lay.off[PK_WS_DQ_ACC];
     char* kr = qr + align_up((size_t)T * Hq * D * 2, 256);

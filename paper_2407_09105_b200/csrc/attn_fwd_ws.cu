@@ -412,6 +412,9 @@ int launch_fwd_ws(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMa
       if (out_dtype == PK_BF16) PK_FWS(128, false, __nv_bfloat16); else PK_FWS(128, false, float);
     }
   }
+  if (rotated) {
+    if (out_dtype == PK_BF16) PK_FWS(64, true, __nv_bfloat16); else PK_FWS(64, true, float);
+  }
   if (out_dtype == PK_BF16) PK_FWS(64, false, __nv_bfloat16);
   PK_FWS(64, false, float);
 #undef PK_FWS
