@@ -151,11 +151,13 @@ int pk_attn_fwd(const void* q, const void* k, const void* v, const int32_t* posi
  * With rope_theta > 0 the gradients are with respect to the un-rotated q and k.
  *   out, out_dtype   the forward's output as it was written
  *   dq [T,Hq,D], dk, dv [T,Hkv,D]   element type grad_dtype (PK_BF16 or PK_F32)
- * Without fused RoPE (rope_theta <= 0) the backward runs as two kernels, one key-block
- * stationary for dK/dV and one query-block stationary for dQ; every gradient is accumulated
- * in a fixed order and is bitwise reproducible.  With fused RoPE one kernel produces all three;
- * dK/dV are still accumulated in a fixed order, dQ goes through fp32 reductions in the
- * workspace (order not fixed) followed by a scale / un-rotate / cast pass.
+ * The backward runs as two kernels, one key-block stationary for dK/dV and one query-block
+ * stationary for dQ; every gradient is accumulated in a fixed order and is bitwise
+ * reproducible.  With rope_theta > 0 they work on rotated copies of q and k (made by a
+ * streaming pass, or left by the forward: PK_REUSE_ROTATED) and rotate dQ / dK back as they
+ * write them.  Only with pk_set_rope_mode(PK_ROPE_IN_TILE) one kernel produces all three and
+ * dQ goes through fp32 reductions in the workspace (order not fixed) followed by a scale /
+ * un-rotate / cast pass.
  */
 int pk_attn_bwd(const void* dout, const void* q, const void* k, const void* v,
                 const void* out, int32_t out_dtype, const float* lse,
