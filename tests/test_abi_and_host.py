@@ -62,6 +62,16 @@ def test_argument_validation_returns_codes_without_a_gpu():
     assert L.pk_seqlens_from_posids_noalloc(1, api.PK_NOALLOC_MAX_TOKENS + 1, 1, None, None,
                                             None) == api.PK_ERR_TOO_LARGE
     assert L.pk_set_timing_events(99, None, None) == api.PK_ERR_INVALID_ARG
+    # packed-stream loss: sizes, strides, dtypes and missing outputs
+    bad = api.PK_ERR_INVALID_ARG
+    assert L.pk_packed_loss_fwd(None, 0, None, -1, 8, 8, -100, None, None, 1, 1, None) == bad
+    assert L.pk_packed_loss_fwd(None, 0, None, 4, 0, 0, -100, None, None, 1, 1, None) == bad
+    assert L.pk_packed_loss_fwd(None, 0, None, 4, 8, 7, -100, None, None, 1, 1, None) == bad     # stride < V
+    assert L.pk_packed_loss_fwd(None, 5, None, 4, 8, 8, -100, None, None, 1, 1, None) == bad     # dtype
+    assert L.pk_packed_loss_fwd(None, 0, None, 4, 8, 8, -100, None, None, None, 1, None) == bad  # no result
+    assert L.pk_packed_loss_fwd(None, 0, None, 4, 8, 8, -100, None, None, 1, 1, None) == bad     # no logits
+    assert L.pk_packed_loss_bwd(None, 0, None, None, None, 1.0, 4, 8, 8, -100, None, None) == bad
+    assert L.pk_packed_loss_bwd(None, 0, None, None, 1, 1.0, 0, 8, 8, -100, None, None) == api.PK_OK  # T = 0
 
 
 def test_assign_streams_balances_by_pairs():
