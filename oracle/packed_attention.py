@@ -136,7 +136,16 @@ def rope(x, position_ids, theta, inverse=False):
 _ROW_BLOCK = 2048   # memory bound only: query rows are independent of each other
 
 
-def _example_head_fwd(q, k, v, scale):
+def _visible(rows, cols, window):
+    """Causal mask of one example, optionally limited to the ``window`` most recent keys
+    (the row's own position included); window <= 0 means no limit."""
+    m = cols <= rows
+    if window > 0:
+        m = m & (cols > rows - window)
+    return m
+
+
+def _example_head_fwd(q, k, v, scale, window=0):
     """q [L, D], k/v [L, D] of ONE example and head -> (O [L, D], lse [L])."""
     L = q.shape[0]
     out = np.empty((L, v.shape[1]), dtype=np.float64)
@@ -146,7 +155,7 @@ def _example_head_fwd(q, k, v, scale):
         s = scale * (q[r0:r1] @ k[:r1].T)                       # keys j <= i only
         rows = np.arange(r0, r1).reshape(-1, 1)
         cols = np.arange(0, r1).reshape(1, -1)
-        s = np.where(cols <= rows, s, -np.inf)                   # causal, diagonal kept
+        s = np.where(_visible(rows, cols, window), s, -np.inf)   # causal, diagonal kept
         m = s.max(axis=1, keepdims=True)
         z = np.exp(s - m).sum(axis=1, keepdims=True)
         l = m + np.log(z)
@@ -156,7 +165,7 @@ def _example_head_fwd(q, k, v, scale):
     return out, lse
 
 
-def _example_head_bwd(do, q, k, v, scale):
+def _example_head_bwd(do, q, k, v, scale, window=0):
     """Gradients of ONE example and head w.r.t. its (already rotated) q, k and v."""
     L = q.shape[0]
     dq = np.zeros_like(q)
@@ -167,7 +176,7 @@ def _example_head_bwd(do, q, k, v, scale):
         s = scale * (q[r0:r1] @ k[:r1].T)
         rows = np.arange(r0, r1).reshape(-1, 1)
         cols = np.arange(0, r1).reshape(1, -1)
-        s = np.where(cols <= rows, s, -np.inf)
+        s = np.where(_visible(rows, cols, window), s, -np.inf)
         m = s.max(axis=1, keepdims=True)
         l = m + np.log(np.exp(s - m).sum(axis=1, keepdims=True))
         p = np.exp(s - l)                                        # masked entries are 0
@@ -185,13 +194,15 @@ def _f64(x):
     return np.asarray(x, dtype=np.float64)
 
 
-def attn_fwd(q, k, v, position_ids, softmax_scale, rope_theta=0.0, examples=None):
+def attn_fwd(q, k, v, position_ids, softmax_scale, rope_theta=0.0, examples=None, window=0):
     """Forward over a packed stream.
 
     q [T, Hq, D], k/v [T, Hkv, D].  Returns (out fp64 [T, Hq, D], lse fp64
     [Hq, T]); lse is the natural log of the sum of exp(scale * q.k) over the
     keys the row may see.  ``examples`` restricts the work to those example
-    indices (other rows are left as NaN).
+    indices (other rows are left as NaN).  ``window`` > 0 limits every row to its
+    ``window`` most recent keys inside its example (sliding-window attention of
+    the Mistral family; the row's own position counts).
     """
     q, k, v = _f64(q), _f64(k), _f64(v)
     T, Hq, D = q.shape
@@ -208,13 +219,14 @@ def attn_fwd(q, k, v, position_ids, softmax_scale, rope_theta=0.0, examples=None
         s, t = int(cu[e]), int(cu[e + 1])
         for h in range(Hq):
             g = h // G
-            o, l = _example_head_fwd(q[s:t, h], k[s:t, g], v[s:t, g], softmax_scale)
+            o, l = _example_head_fwd(q[s:t, h], k[s:t, g], v[s:t, g], softmax_scale, window)
             out[s:t, h] = o
             lse[h, s:t] = l
     return out, lse
 
 
-def attn_bwd(dout, q, k, v, position_ids, softmax_scale, rope_theta=0.0, examples=None):
+def attn_bwd(dout, q, k, v, position_ids, softmax_scale, rope_theta=0.0, examples=None,
+             window=0):
     """Backward over a packed stream: (dq [T,Hq,D], dk, dv [T,Hkv,D]) in fp64.
 
     dK and dV of a kv head are summed over the G query heads that read it.  With
@@ -240,7 +252,7 @@ def attn_bwd(dout, q, k, v, position_ids, softmax_scale, rope_theta=0.0, example
         for h in range(Hq):
             g = h // G
             a, b, c = _example_head_bwd(dout[s:t, h], q[s:t, h], k[s:t, g], v[s:t, g],
-                                        softmax_scale)
+                                        softmax_scale, window)
             dq[s:t, h] = a
             dk[s:t, g] += b
             dv[s:t, g] += c

@@ -440,3 +440,71 @@ def test_examples_subset_argument():
     g1 = orc.attn_bwd(do, q, k, v, pos, 0.5, examples=[2])
     for a, b in zip(g, g1):
         assert np.array_equal(a[9:], b[9:]) and np.isnan(b[:9]).all()
+
+
+# ---------------------------------------------------------------- sliding window
+
+def _dense_window_mask(pos, window):
+    """Dense mask written out by hand: same example, key not after the query, and (window > 0)
+    at most window - 1 positions before it."""
+    pos = np.asarray(pos)
+    T = len(pos)
+    ex = np.zeros(T, dtype=np.int64)
+    for t in range(1, T):
+        ex[t] = ex[t - 1] + (1 if pos[t] <= pos[t - 1] else 0)
+    m = np.zeros((T, T), dtype=bool)
+    for i in range(T):
+        for j in range(T):
+            m[i, j] = ex[i] == ex[j] and j <= i and (window <= 0 or i - j < window)
+    return m
+
+
+@pytest.mark.parametrize("window", [1, 2, 3, 5, 100])
+def test_sliding_window_against_torch_sdpa_and_autograd(window):
+    rng = np.random.default_rng(20 + window)
+    lens = [7, 1, 9, 4]
+    T, Hq, Hkv, D = sum(lens), 4, 2, 8
+    G = Hq // Hkv
+    q = rng.standard_normal((T, Hq, D))
+    k = rng.standard_normal((T, Hkv, D))
+    v = rng.standard_normal((T, Hkv, D))
+    do = rng.standard_normal((T, Hq, D))
+    pos = wl.position_ids_from_lengths(lens)
+    mask = _dense_window_mask(pos, window)
+    tq, tk, tv = (torch.from_numpy(x).clone().requires_grad_(True) for x in (q, k, v))
+    o = torch.nn.functional.scaled_dot_product_attention(
+        tq.permute(1, 0, 2)[None], tk.repeat_interleave(G, dim=1).permute(1, 0, 2)[None],
+        tv.repeat_interleave(G, dim=1).permute(1, 0, 2)[None], attn_mask=torch.from_numpy(mask),
+        scale=0.6)[0].permute(1, 0, 2)
+    (o * torch.from_numpy(do)).sum().backward()
+    oo, ll = orc.attn_fwd(q, k, v, pos, 0.6, window=window)
+    assert np.allclose(oo, o.detach().numpy(), atol=1e-12)
+    dq, dk, dv = orc.attn_bwd(do, q, k, v, pos, 0.6, window=window)
+    assert np.allclose(dq, tq.grad.numpy(), atol=1e-11)
+    assert np.allclose(dk, tk.grad.numpy(), atol=1e-11)
+    assert np.allclose(dv, tv.grad.numpy(), atol=1e-11)
+    # the row sees min(window, position + 1) keys: lse of all-zero scores would be its log
+    z, lz = orc.attn_fwd(np.zeros_like(q), k, v, pos, 0.6, window=window)
+    seen = np.minimum(window, np.asarray(pos) + 1)
+    assert np.allclose(lz, np.log(seen)[None, :].repeat(Hq, 0), atol=1e-12)
+
+
+def test_sliding_window_special_cases():
+    rng = np.random.default_rng(30)
+    lens = [6, 10]
+    T, H, D = sum(lens), 2, 4
+    q, k, v = (rng.standard_normal((T, H, D)) for _ in range(3))
+    pos = wl.position_ids_from_lengths(lens)
+    # window 1: every row sees itself only -> out = v, lse = its own score
+    o, l = orc.attn_fwd(q, k, v, pos, 0.5, window=1)
+    assert np.allclose(o, v, atol=1e-14)
+    assert np.allclose(l, 0.5 * np.einsum("thd,thd->ht", q, k), atol=1e-13)
+    # a window at least as long as the longest example changes nothing; 0 means no window
+    a, la = orc.attn_fwd(q, k, v, pos, 0.5)
+    for wdw in (10, 11, 1000, 0):
+        b, lb = orc.attn_fwd(q, k, v, pos, 0.5, window=wdw)
+        assert np.array_equal(a, b) and np.array_equal(la, lb)
+    # with rope: the window is over positions inside the example, like the mask
+    c, _ = orc.attn_fwd(q, k, v, pos, 0.5, 1e4, window=3)
+    d, _ = orc.attn_fwd(orc.rope(q, pos, 1e4), orc.rope(k, pos, 1e4), v, pos, 0.5, window=3)
+    assert np.allclose(c, d, atol=1e-13)
