@@ -135,15 +135,15 @@ def _time_oracle(w: wl.Workload, steps: int = 1):
         threads = len(os.sched_getaffinity(0))
     lens = _oracle_sample(w)
     sw = wl.Workload(w.name + "_sample", w.seed, w.num_q_heads, w.num_kv_heads, w.head_dim,
-                     w.rope_theta, [lens], w.packing)
+                     w.rope_theta, [lens], w.packing, w.window)
     st = wl.stream_tensors(sw, lens, 0, "cpu")
     q, k, v, do = (x.to(torch.float64).numpy() for x in (st.q, st.k, st.v, st.dout))
     pos = st.position_ids.numpy()
     best = None
     for _ in range(steps):
         t0 = time.perf_counter()
-        orc.attn_fwd(q, k, v, pos, sw.softmax_scale, sw.rope_theta)
-        orc.attn_bwd(do, q, k, v, pos, sw.softmax_scale, sw.rope_theta)
+        orc.attn_fwd(q, k, v, pos, sw.softmax_scale, sw.rope_theta, window=w.window)
+        orc.attn_bwd(do, q, k, v, pos, sw.softmax_scale, sw.rope_theta, window=w.window)
         dt = time.perf_counter() - t0
         best = dt if best is None else min(best, dt)
     flops = sw.useful_flops_fwd + sw.useful_flops_bwd
@@ -301,6 +301,8 @@ def main():
                     help="use only the first N packs of the workload (small cases for profiling)")
     ap.add_argument("--per-stream", action="store_true",
                     help="one call per pack / mini-batch instead of one flat stream")
+    ap.add_argument("--window", type=int, default=0,
+                    help="sliding-window attention: keys visible per row (0 = all, the default)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -313,6 +315,9 @@ def main():
     if args.packs > 0:
         w = wl.Workload(f"{w.name}[:{args.packs}]", w.seed, w.num_q_heads, w.num_kv_heads,
                         w.head_dim, w.rope_theta, w.streams[:args.packs], w.packing)
+    if args.window > 0:
+        w = wl.Workload(f"{w.name}+window{args.window}", w.seed, w.num_q_heads, w.num_kv_heads,
+                        w.head_dim, w.rope_theta, w.streams, w.packing, args.window)
     if args.impl == "reference":
         run_reference(args, w)
         return
@@ -357,18 +362,18 @@ def main():
         def step():
             for (q_, k_, v_, do_, pos_, out_, lse_, dq_, dk_, dv_) in pieces:
                 api.pk_attn_fwd(q_, k_, v_, pos_, scale, theta, out_, lse_, ws,
-                                reuse_plan=False, stream=stream)
+                                reuse_plan=False, window=w.window, stream=stream)
                 api.pk_attn_bwd(do_, q_, k_, v_, out_, lse_, pos_, scale, theta,
-                                dq_, dk_, dv_, ws, reuse_plan=True, reuse_rotated=True, stream=stream)
+                                dq_, dk_, dv_, ws, reuse_plan=True, reuse_rotated=True, window=w.window, stream=stream)
         calls_per_step = len(pieces)
     else:
         ws = api.alloc_workspace(T, Hq, Hkv, D)
 
         def step():
             api.pk_attn_fwd(st.q, st.k, st.v, st.position_ids, scale, theta, out, lse, ws,
-                            reuse_plan=False, stream=stream)
+                            reuse_plan=False, window=w.window, stream=stream)
             api.pk_attn_bwd(st.dout, st.q, st.k, st.v, out, lse, st.position_ids, scale, theta,
-                            dq, dk, dv, ws, reuse_plan=True, reuse_rotated=True, stream=stream)
+                            dq, dk, dv, ws, reuse_plan=True, reuse_rotated=True, window=w.window, stream=stream)
         calls_per_step = 1
 
     def barrier():
@@ -440,10 +445,10 @@ def main():
             def compute(i, s):
                 a, b = spans[i]
                 api.pk_attn_fwd(st.q[a:b], st.k[a:b], st.v[a:b], st.position_ids[a:b], scale, theta,
-                                out[a:b], lse_p[i], ws_p, reuse_plan=False, stream=s)
+                                out[a:b], lse_p[i], ws_p, reuse_plan=False, window=w.window, stream=s)
                 api.pk_attn_bwd(st.dout[a:b], st.q[a:b], st.k[a:b], st.v[a:b], out[a:b], lse_p[i],
                                 st.position_ids[a:b], scale, theta, dq[a:b], dk[a:b], dv[a:b], ws_p,
-                                reuse_plan=True, reuse_rotated=True, stream=s)
+                                reuse_plan=True, reuse_rotated=True, window=w.window, stream=s)
 
             pipe = pipeline.HostPipeline(cut(host_in), cut(dev_in), cut(dev_out), cut(host_out), compute)
 
@@ -516,7 +521,7 @@ def main():
         "config": {"workload": (f"{w.name}: {w.packing}, {len(w.streams)} packs, " +
                                 ("one call per pack" if args.per_stream else "as one flat stream")),
                    "tokens": T, "examples": len(lens), "Hq": Hq, "Hkv": Hkv, "head_dim": D,
-                   "rope_theta": theta, "causal_pairs": w.causal_pairs,
+                   "rope_theta": theta, "window": w.window, "causal_pairs": w.causal_pairs,
                    "flop_convention": "14*D*Hq*sum L(L+1)/2", "l2": "inputs_exceed_l2",
                    "replicas": world},
         "tokens_per_s": tokens_per_s,

@@ -125,6 +125,12 @@ int pk_rope_apply(void* x, const int32_t* position_ids, int32_t T, int32_t H, in
  *   q, k, v       bf16
  *   rope_theta    > 0: q and k are rotated by position_ids while their tiles are loaded
  *                 (q', k'); <= 0: q and k are used as given
+ *   window        0: every row sees all keys of its example up to itself.  > 0: only its `window`
+ *                 most recent keys, its own position included (sliding-window attention of
+ *                 the Mistral family; the paper lists the model, the definition is that
+ *                 model's).  Key tiles that no row of a query block can see are skipped.
+ *                 Not available with pk_set_rope_mode(PK_ROPE_IN_TILE) and rope_theta > 0
+ *                 (PK_ERR_UNSUPPORTED); pk_attn_bwd must be given the forward's value.
  *   out           [T, Hq, D], element type out_dtype (PK_BF16 or PK_F32)
  *   lse           fp32 [Hq, T]
  *   reuse_plan    bit mask.  0: run the planning step of pk_seqlens_from_posids first (same
@@ -139,7 +145,7 @@ int pk_rope_apply(void* x, const int32_t* position_ids, int32_t T, int32_t H, in
 #define PK_REUSE_ROTATED  2
 int pk_attn_fwd(const void* q, const void* k, const void* v, const int32_t* position_ids,
                 int32_t T, int32_t Hq, int32_t Hkv, int32_t D,
-                float softmax_scale, float rope_theta,
+                float softmax_scale, float rope_theta, int32_t window,
                 void* out, int32_t out_dtype, float* lse,
                 int32_t reuse_plan, void* workspace, size_t workspace_bytes, void* stream);
 
@@ -163,7 +169,7 @@ int pk_attn_bwd(const void* dout, const void* q, const void* k, const void* v,
                 const void* out, int32_t out_dtype, const float* lse,
                 const int32_t* position_ids,
                 int32_t T, int32_t Hq, int32_t Hkv, int32_t D,
-                float softmax_scale, float rope_theta,
+                float softmax_scale, float rope_theta, int32_t window,
                 void* dq, void* dk, void* dv, int32_t grad_dtype,
                 int32_t reuse_plan, void* workspace, size_t workspace_bytes, void* stream);
 

@@ -43,10 +43,10 @@ _SIGNATURES = {
                                             ctypes.POINTER(_sz), ctypes.POINTER(_sz)]),
     "pk_seqlens_from_posids": (ctypes.c_int, [_vp, _i32, _vp, _vp, _vp, _vp, _sz, _vp]),
     "pk_rope_apply": (ctypes.c_int, [_vp, _vp, _i32, _i32, _i32, _f32, _i32, _vp]),
-    "pk_attn_fwd": (ctypes.c_int, [_vp, _vp, _vp, _vp, _i32, _i32, _i32, _i32, _f32, _f32,
+    "pk_attn_fwd": (ctypes.c_int, [_vp, _vp, _vp, _vp, _i32, _i32, _i32, _i32, _f32, _f32, _i32,
                                    _vp, _i32, _vp, _i32, _vp, _sz, _vp]),
     "pk_attn_bwd": (ctypes.c_int, [_vp, _vp, _vp, _vp, _vp, _i32, _vp, _vp,
-                                   _i32, _i32, _i32, _i32, _f32, _f32,
+                                   _i32, _i32, _i32, _i32, _f32, _f32, _i32,
                                    _vp, _vp, _vp, _i32, _i32, _vp, _sz, _vp]),
     "pk_status_read": (ctypes.c_int, [_vp, _vp, ctypes.POINTER(_i32), ctypes.POINTER(_i32)]),
     "pk_set_timing_events": (ctypes.c_int, [_i32, _vp, _vp]),
@@ -175,20 +175,24 @@ def pk_rope_apply(x: torch.Tensor, position_ids: torch.Tensor, theta: float,
 
 def pk_attn_fwd(q, k, v, position_ids, softmax_scale: float, rope_theta: float,
                 out: torch.Tensor, lse: torch.Tensor, workspace: torch.Tensor,
-                reuse_plan: bool = False, stream=None) -> None:
+                reuse_plan: bool = False, window: int = 0, stream=None) -> None:
+    """``window`` > 0: sliding-window attention (each row sees its ``window`` most recent keys)."""
     T, Hq, D = q.shape
     Hkv = k.shape[1]
     _check("pk_attn_fwd",
            lib().pk_attn_fwd(_ptr(q), _ptr(k), _ptr(v), _ptr(position_ids), T, Hq, Hkv, D,
-                             softmax_scale, rope_theta, _ptr(out), _dtype_code(out), _ptr(lse),
-                             int(reuse_plan), _ptr(workspace), workspace.numel(), _stream(stream)))
+                             softmax_scale, rope_theta, int(window), _ptr(out), _dtype_code(out),
+                             _ptr(lse), int(reuse_plan), _ptr(workspace), workspace.numel(),
+                             _stream(stream)))
 
 
 def pk_attn_bwd(dout, q, k, v, out, lse, position_ids, softmax_scale: float, rope_theta: float,
                 dq: torch.Tensor, dk: torch.Tensor, dv: torch.Tensor, workspace: torch.Tensor,
-                reuse_plan: bool = True, reuse_rotated: bool = False, stream=None) -> None:
+                reuse_plan: bool = True, reuse_rotated: bool = False, window: int = 0,
+                stream=None) -> None:
     """``reuse_rotated``: the rotated q / k copies the forward left in ``workspace`` are still
-    valid (same q, k, position_ids, rope_theta; workspace untouched since)."""
+    valid (same q, k, position_ids, rope_theta; workspace untouched since).  ``window``: the
+    forward's sliding window (0 = none)."""
     T, Hq, D = q.shape
     Hkv = k.shape[1]
     if not (dq.dtype == dk.dtype == dv.dtype):
@@ -196,7 +200,7 @@ def pk_attn_bwd(dout, q, k, v, out, lse, position_ids, softmax_scale: float, rop
     _check("pk_attn_bwd",
            lib().pk_attn_bwd(_ptr(dout), _ptr(q), _ptr(k), _ptr(v), _ptr(out), _dtype_code(out),
                              _ptr(lse), _ptr(position_ids), T, Hq, Hkv, D, softmax_scale,
-                             rope_theta, _ptr(dq), _ptr(dk), _ptr(dv), _dtype_code(dq),
+                             rope_theta, int(window), _ptr(dq), _ptr(dk), _ptr(dv), _dtype_code(dq),
                              (PK_REUSE_PLAN if reuse_plan else 0) |
                              (PK_REUSE_ROTATED if reuse_rotated else 0),
                              _ptr(workspace), workspace.numel(), _stream(stream)))

@@ -483,13 +483,17 @@ int launch_bwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& 
 extern "C" int pk_attn_bwd(const void* dout, const void* q, const void* k, const void* v,
                            const void* out, int32_t out_dtype, const float* lse,
                            const int32_t* position_ids, int32_t T, int32_t Hq, int32_t Hkv,
-                           int32_t D, float softmax_scale, float rope_theta, void* dq, void* dk,
-                           void* dv, int32_t grad_dtype, int32_t reuse_plan, void* workspace,
+                           int32_t D, float softmax_scale, float rope_theta, int32_t window,
+                           void* dq, void* dk, void* dv, int32_t grad_dtype,
+                           int32_t reuse_plan, void* workspace,
                            size_t workspace_bytes, void* stream_) {
   using namespace pk;
   cudaStream_t stream = static_cast<cudaStream_t>(stream_);
-  if (T < 0 || Hq <= 0 || Hkv <= 0 || !(softmax_scale > 0.f)) return PK_ERR_INVALID_ARG;
+  if (T < 0 || Hq <= 0 || Hkv <= 0 || !(softmax_scale > 0.f) || window < 0)
+    return PK_ERR_INVALID_ARG;
   if (!shape_supported(T, Hq, Hkv, D)) return PK_ERR_UNSUPPORTED;
+  if (window > 0 && rope_theta > 0.f && g_rope_mode != PK_ROPE_ROTATED_COPIES)
+    return PK_ERR_UNSUPPORTED;
   if ((out_dtype != PK_BF16 && out_dtype != PK_F32) ||
       (grad_dtype != PK_BF16 && grad_dtype != PK_F32))
     return PK_ERR_UNSUPPORTED;
@@ -563,12 +567,12 @@ extern "C" int pk_attn_bwd(const void* dout, const void* q, const void* k, const
     if (!make_tile_map_bf16(&tqr, qr, T, Hq * D) || !make_tile_map_bf16(&tkr, kr, T, Hkv * D))
       return PK_ERR_CUDA;
     return launch_bwd_ws(tqr, tkr, tv, tdo, ws, lay, lse, dq, dk, dv, T, Hq, Hkv, D, grad_dtype,
-                         softmax_scale, true, stream);
+                         softmax_scale, window, true, stream);
   }
   if (!use_rope) {
     // two warp-specialised kernels (dK/dV, then dQ); dQ is final, no finishing pass
     return launch_bwd_ws(tq, tk, tv, tdo, ws, lay, lse, dq, dk, dv, T, Hq, Hkv, D, grad_dtype,
-                         softmax_scale, false, stream);
+                         softmax_scale, window, false, stream);
   } else {
 #define PK_BWD(DD, RR, TT)                                                                      \
   rc = launch_bwd<DD, RR, TT>(tq, tk, tv, tdo, ws, lay, lse, dk, dv, T, Hq, Hkv, softmax_scale, \

@@ -99,7 +99,7 @@ attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     const float* __restrict__ lse, const float* __restrict__ delta,
                     GradT* __restrict__ dk, GradT* __restrict__ dv,
                     const float2* __restrict__ rope_table,
-                    int T, int Hq, int Hkv, float scale, float scale_log2) {
+                    int T, int Hq, int Hkv, float scale, float scale_log2, int window) {
   using L = DkvSmem<D>;
   extern __shared__ __align__(1024) uint8_t smem[];
   const uint32_t sbase = smem_u32(smem);
@@ -149,6 +149,12 @@ attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   const bool plan_ok = (hdr[PK_HDR_PLAN_T] == T);
   if (!plan_ok && blockIdx.x == 0 && tid == 0) set_status(hdr, PK_ERR_NO_PLAN, T);
   const int n_units = plan_ok ? hdr[PK_HDR_N_ITEMS] * Hkv : 0;
+  // query tiles of a key block: to the example's end, or (sliding window) to the last query that
+  // still sees the block's last key, window - 1 rows further down
+  auto query_tiles = [&](int kv_len, int q_len) {
+    const int n = (q_len + kBM - 1) / kBM;
+    return window > 0 ? min(n, (kv_len - 1 + window - 1) / kBM + 1) : n;
+  };
 
   if (warp == kLoadWarp) {
     // =============================== loader ===============================================
@@ -175,7 +181,7 @@ attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       const int4 it = items[order[u / Hkv]];
       const int g = u % Hkv;
       const int kv_start = it.x, q_start = it.z, q_len = it.w;
-      const int n_q = (q_len + kBM - 1) / kBM;
+      const int n_q = query_tiles(it.y, q_len);
       mbar_wait(bar(kvKvEmpty), (uc & 1) ^ 1, s_abort);
       if (lane == 0) {
         mbar_expect_tx(bar(kvKvFull), 2 * L::kTileBytes);
@@ -273,7 +279,7 @@ attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         const int u = s_unit[uc % kUnitRing];
         if (u >= n_units || *s_abort) break;
         const int4 it = items[order[u / Hkv]];
-        const int n_q = (it.w + kBM - 1) / kBM;
+        const int n_q = query_tiles(it.y, it.w);
         const int n_steps = G * n_q;
         mbar_wait(bar(kvKvFull), uc & 1, s_abort);
         // prologue: S(0) goes where dP of the previous unit's last step was, so that one must
@@ -343,11 +349,15 @@ attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       const int4 it = items[order[u / Hkv]];
       const int g = u % Hkv;
       const int kv_start = it.x, kv_len = it.y, q_len = it.w;
-      const int n_q = (q_len + kBM - 1) / kBM;
+      const int n_q = query_tiles(kv_len, q_len);
       for (int hh = 0; hh < G; ++hh) {
         for (int i = 0; i < n_q; ++i, ++gs) {
           const int sl = gs & 1;
-          const int q_left = q_len - i * kBM;
+          // queries [i*128, ..) of the unit: up to the example's end and, with a sliding window,
+          // less than `window` rows below this thread's key
+          const int q_rows = q_len - i * kBM;
+          const int q_left = window > 0 ? min(q_rows, row + window - i * kBM) : q_rows;
+          const bool win_edge = window > 0 && (i + 1) * kBM > window;
           const int col_min = (i == 0) ? row : 0;
           const uint32_t tA = region_s(gs) + lane_off + col0;    // S^T, then P^T | dS^T
           const uint32_t tB = region_dp(gs) + lane_off + col0;   // dP^T
@@ -370,7 +380,7 @@ attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
               p[c + 3] = fast_exp2(fmaf(__uint_as_float(sv[c + 3]), scale_log2, -l4.w));
             }
           }
-          if (i == 0 || q_left < kBM) {   // diagonal tile or last, partial tile; interior tiles skip this
+          if (i == 0 || q_rows < kBM || win_edge) {   // diagonal, last partial or window-edge tile; interior tiles skip this
 #pragma unroll
             for (int c = 0; c < 64; ++c) {
               const int col = col0 + c;
@@ -512,7 +522,7 @@ attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                    const int4* __restrict__ items, const int32_t* __restrict__ order, int32_t* hdr,
                    const float* __restrict__ lse, const float* __restrict__ delta,
                    GradT* __restrict__ dq, const float2* __restrict__ rope_table, int T, int Hq,
-                   int Hkv, float scale, float scale_log2) {
+                   int Hkv, float scale, float scale_log2, int window) {
   using L = DqSmem<D>;
   extern __shared__ __align__(1024) uint8_t smem[];
   const uint32_t sbase = smem_u32(smem);
@@ -555,6 +565,12 @@ attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
   const int G = Hq / Hkv;
   const bool plan_ok = (hdr[PK_HDR_PLAN_T] == T);
   const int n_units = plan_ok ? hdr[PK_HDR_N_ITEMS] * Hq : 0;
+  // first key tile of a query block: 0, or (sliding window) the tile holding the key window - 1
+  // positions before the block's first row
+  auto first_key_tile = [&](int q_start, int kv_start) {
+    const int reach = q_start - (window - 1) - kv_start;
+    return (window > 0 && reach > 0) ? reach / kBN : 0;
+  };
 
   if (warp == kLoadWarp) {
     // =============================== loader ===============================================
@@ -573,6 +589,7 @@ attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         const int h = u % Hq, g = h / G;
         const int q_start = it.x, kv_start = it.z, kv_len = it.w;
         const int n_kv = (kv_len + kBN - 1) / kBN;
+        const int j0 = first_key_tile(q_start, kv_start);
         mbar_wait(bar(dqQEmpty), (uc & 1) ^ 1, s_abort);
         mbar_expect_tx(bar(dqQFull), 2 * L::kTileBytes);
 #pragma unroll
@@ -580,7 +597,7 @@ attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
           tma_load_2d(sbase + L::kQ + b * L::kBoxBytes, &tm_q, h * D + b * 64, q_start, bar(dqQFull));
           tma_load_2d(sbase + L::kdO + b * L::kBoxBytes, &tm_do, h * D + b * 64, q_start, bar(dqQFull));
         }
-        for (int j = 0; j < n_kv; ++j, ++gk) {
+        for (int j = j0; j < n_kv; ++j, ++gk) {
           const int ks = gk % L::kKStages, vs = gk % L::kVStages;
           const uint32_t sK = sbase + L::kK0 + ks * L::kTileBytes;
           const uint32_t sV = sbase + L::kV0 + vs * L::kTileBytes;
@@ -648,12 +665,13 @@ attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         if (u >= n_units || *s_abort) break;
         const int4 it = items[order[u / Hq]];
         const int n_kv = (it.w + kBN - 1) / kBN;
+        const int j0 = first_key_tile(it.x, it.z);
         mbar_wait(bar(dqQtReady), uc & 1, s_abort);
         if (gk > 0) mbar_wait(bar(dqSRead), (gk - 1) & 1, s_abort);   // S of the previous step read
         tc_fence_after();
         issue_s(gk);
         issue_dp(gk);
-        for (int j = 0; j < n_kv; ++j, ++gk) {
+        for (int j = j0; j < n_kv; ++j, ++gk) {
           const int ks = gk % L::kKStages;
           const uint32_t k_lo = desc_lo(sbase + L::kK0 + ks * L::kTileBytes, L::kBoxBytes);
           const bool more = (j + 1 < n_kv);
@@ -662,13 +680,13 @@ attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             issue_s(gk + 1);
           }
           mbar_wait(bar(dqDsReady), gk & 1, s_abort);
-          if (j == 0 && uc > 0) mbar_wait(bar(dqRead), (uc - 1) & 1, s_abort);
+          if (j == j0 && uc > 0) mbar_wait(bar(dqRead), (uc - 1) & 1, s_abort);
           tc_fence_after();
           if (leader) {
 #pragma unroll
             for (int kk = 0; kk < kBN / 16; ++kk)   // dQ += dS K   (dS of keys 16kk.. : see compute)
               mma_ts(tdQ, tdP + (kk / (kCW / 16)) * kCW + (kk % (kCW / 16)) * 8,
-                     desc_from_lo(k_lo + ((kk * 2048) >> 4)), kIdescDQ, (j > 0) | (kk > 0));
+                     desc_from_lo(k_lo + ((kk * 2048) >> 4)), kIdescDQ, (j > j0) | (kk > 0));
             mma_commit(bar(dqKEmpty0 + ks));
           }
           __syncwarp();
@@ -722,11 +740,12 @@ attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
       const int h = u % Hq;
       const int q_start = it.x, q_len = it.y, kv_len = it.w;
       const int n_kv = (kv_len + kBN - 1) / kBN;
+      const int j0 = first_key_tile(q_start, it.z);
       const int tok = q_start + row;
       const float lse2 = (tok < T) ? lse[(size_t)h * T + tok] * kLog2eWs : 0.f;
       const float dl = (tok < T) ? delta[(size_t)h * T + tok] : 0.f;
 
-      for (int j = 0; j < n_kv; ++j, ++gk) {
+      for (int j = j0; j < n_kv; ++j, ++gk) {
         mbar_wait(bar(dqSFull), gk & 1, s_abort);
         tc_fence_after();
         float p[kCW];
@@ -744,6 +763,13 @@ attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
 #pragma unroll
             for (int c = 0; c < kCW; ++c)
               if (qd * kCW + c > row) p[c] = 0.f;
+          }
+          // sliding window: keys more than window - 1 before the row
+          const int lo = (window > 0) ? (q_start + row - (window - 1) - it.z - j * kBN) : 0;
+          if (lo > 0) {
+#pragma unroll
+            for (int c = 0; c < kCW; ++c)
+              if (qd * kCW + c < lo) p[c] = 0.f;
           }
         }
         mbar_wait(bar(dqDpFull), gk & 1, s_abort);
@@ -830,7 +856,7 @@ attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
 template <int D, bool kRot, typename GradT>
 int launch_ws(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
               const CUtensorMap& tdo, char* ws, const WorkspaceLayout& lay, const float* lse,
-              void* dq, void* dk, void* dv, int T, int Hq, int Hkv, float scale,
+              void* dq, void* dk, void* dv, int T, int Hq, int Hkv, float scale, int window,
               cudaStream_t stream) {
   auto kern_kv = attn_bwd_dkv_kernel<D, kRot, GradT>;
   auto kern_q = attn_bwd_dq_kernel<D, kRot, GradT>;
@@ -853,7 +879,7 @@ int launch_ws(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& t
         tq, tk, tv, tdo, reinterpret_cast<const int4*>(ws + lay.off[PK_WS_BWD_ITEMS]),
         reinterpret_cast<const int32_t*>(ws + lay.off[PK_WS_BWD_ORDER]), hdr, lse, delta,
         static_cast<GradT*>(dk), static_cast<GradT*>(dv), table, T, Hq, Hkv, scale,
-        scale * kLog2eWs);
+        scale * kLog2eWs, window);
   }
   if (launch_status() != PK_OK) return PK_ERR_CUDA;
   {
@@ -861,7 +887,7 @@ int launch_ws(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& t
     kern_q<<<grid, kWsThreads, DqSmem<D>::kTotal, stream>>>(
         tq, tk, tv, tdo, reinterpret_cast<const int4*>(ws + lay.off[PK_WS_FWD_ITEMS]),
         reinterpret_cast<const int32_t*>(ws + lay.off[PK_WS_FWD_ORDER]), hdr, lse, delta,
-        static_cast<GradT*>(dq), table, T, Hq, Hkv, scale, scale * kLog2eWs);
+        static_cast<GradT*>(dq), table, T, Hq, Hkv, scale, scale * kLog2eWs, window);
   }
   return launch_status();
 }
@@ -871,10 +897,10 @@ int launch_ws(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& t
 int launch_bwd_ws(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
                   const CUtensorMap& tdo, char* ws, const WorkspaceLayout& lay, const float* lse,
                   void* dq, void* dk, void* dv, int T, int Hq, int Hkv, int D, int grad_dtype,
-                  float scale, bool rotated, cudaStream_t stream) {
+                  float scale, int window, bool rotated, cudaStream_t stream) {
 #define PK_BWS(DD, RR, TT)                                                                     \
   return launch_ws<DD, RR, TT>(tq, tk, tv, tdo, ws, lay, lse, dq, dk, dv, T, Hq, Hkv, scale, \
-                               stream)
+                               window, stream)
   if (D == 128) {
     if (rotated) {
       if (grad_dtype == PK_BF16) PK_BWS(128, true, __nv_bfloat16); else PK_BWS(128, true, float);

@@ -334,13 +334,18 @@ int launch_fwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& 
 
 extern "C" int pk_attn_fwd(const void* q, const void* k, const void* v,
                            const int32_t* position_ids, int32_t T, int32_t Hq, int32_t Hkv,
-                           int32_t D, float softmax_scale, float rope_theta, void* out,
-                           int32_t out_dtype, float* lse, int32_t reuse_plan, void* workspace,
+                           int32_t D, float softmax_scale, float rope_theta, int32_t window,
+                           void* out, int32_t out_dtype, float* lse, int32_t reuse_plan,
+                           void* workspace,
                            size_t workspace_bytes, void* stream_) {
   using namespace pk;
   cudaStream_t stream = static_cast<cudaStream_t>(stream_);
-  if (T < 0 || Hq <= 0 || Hkv <= 0 || !(softmax_scale > 0.f)) return PK_ERR_INVALID_ARG;
+  if (T < 0 || Hq <= 0 || Hkv <= 0 || !(softmax_scale > 0.f) || window < 0)
+    return PK_ERR_INVALID_ARG;
   if (!shape_supported(T, Hq, Hkv, D)) return PK_ERR_UNSUPPORTED;
+  // the sliding window lives in the warp-specialised kernels only
+  if (window > 0 && rope_theta > 0.f && g_rope_mode != PK_ROPE_ROTATED_COPIES)
+    return PK_ERR_UNSUPPORTED;
   if (out_dtype != PK_BF16 && out_dtype != PK_F32) return PK_ERR_UNSUPPORTED;
   if (workspace == nullptr || (reinterpret_cast<uintptr_t>(workspace) & 255u) != 0)
     return PK_ERR_INVALID_ARG;
@@ -370,7 +375,7 @@ extern "C" int pk_attn_fwd(const void* q, const void* k, const void* v,
         !make_tile_map_bf16(&tvv, v, T, Hkv * D))
       return PK_ERR_CUDA;
     return launch_fwd_ws(tqr, tkr, tvv, ws, lay, out, lse, T, Hq, Hkv, D, out_dtype, softmax_scale,
-                         true, stream);
+                         window, true, stream);
   }
   if (use_rope) {
     int rc = rope_table_launch(position_ids, T, D, rope_theta,
@@ -384,7 +389,7 @@ extern "C" int pk_attn_fwd(const void* q, const void* k, const void* v,
 
   if (!use_rope)   // two tiles per CTA (two heads of a kv head, or two query blocks), warp-specialised
     return launch_fwd_ws(tq, tk, tv, ws, lay, out, lse, T, Hq, Hkv, D, out_dtype, softmax_scale,
-                         false, stream);
+                         window, false, stream);
 #define PK_FWD(DD, RR, TT) \
   return launch_fwd<DD, RR, TT>(tq, tk, tv, ws, lay, out, lse, T, Hq, Hkv, softmax_scale, stream)
   if (D == 128) {

@@ -77,10 +77,11 @@ __device__ __forceinline__ void store_out32(OutT* dst, const uint32_t* r, float 
 struct FwdUnit {
   int h[2], q_start[2], q_len[2], diag[2];   // per tile: head, rows, rows to store, diagonal step
   int g, kv_start, n_kv;
+  int j0;                                    // first key step (> 0 only with a sliding window)
 };
 __device__ __forceinline__ FwdUnit decode_fwd_unit(int u, const int4* __restrict__ items,
                                                    const int32_t* __restrict__ order, int Hq,
-                                                   int G, bool pair_blocks) {
+                                                   int G, bool pair_blocks, int window) {
   FwdUnit w;
   if (!pair_blocks) {
     const int pairs = Hq / 2;
@@ -105,6 +106,10 @@ __device__ __forceinline__ FwdUnit decode_fwd_unit(int u, const int4* __restrict
     if (b >= 1) { w.q_start[0] = it.x - kBM; w.q_len[0] = kBM; w.diag[0] = b - 1; }
     else        { w.q_start[0] = it.x;       w.q_len[0] = 0;   w.diag[0] = 0; }
   }
+  // sliding window: the first row of tile 0 reaches back window - 1 keys; whole key tiles
+  // before that are skipped (rows further down see even less of them: masked in the softmax)
+  const int reach = w.q_start[0] - (window - 1) - w.kv_start;
+  w.j0 = (window > 0 && reach > 0) ? reach / kBN : 0;
   return w;
 }
 // block-pair mode: item n leads a unit when an even number of blocks follows it in its example
@@ -121,7 +126,7 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                    const __grid_constant__ CUtensorMap tm_v, const int4* __restrict__ items,
                    const int4* __restrict__ bwd_items, const int32_t* __restrict__ order,
                    int32_t* hdr, OutT* __restrict__ out, float* __restrict__ lse, int T, int Hq,
-                   int Hkv, float scale_log2) {
+                   int Hkv, float scale_log2, int window) {
   using L = FwsSmem<D>;
   extern __shared__ __align__(1024) uint8_t smem[];
   const uint32_t sbase = smem_u32(smem);
@@ -182,8 +187,8 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         s_unit[uc % kFwsUnitRing] = u;
         mbar_arrive(bar(fUnitFull0 + uc % kFwsUnitRing));
         if (u >= n_units || *s_abort) break;
-        const FwdUnit w = decode_fwd_unit(u, items, order, Hq, G, pair_blocks);
-        const int g = w.g, kv_start = w.kv_start, n_kv = w.n_kv;
+        const FwdUnit w = decode_fwd_unit(u, items, order, Hq, G, pair_blocks, window);
+        const int g = w.g, kv_start = w.kv_start, n_kv = w.n_kv, j0 = w.j0;
         mbar_wait(bar(fQEmpty), (uc & 1) ^ 1, s_abort);
         mbar_expect_tx(bar(fQFull), 2 * L::kTileBytes);
 #pragma unroll
@@ -192,7 +197,7 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
           for (int b = 0; b < L::kBoxes; ++b)
             tma_load_2d(sbase + L::kQ0 + t * L::kTileBytes + b * L::kBoxBytes, &tm_q,
                         w.h[t] * D + b * 64, w.q_start[t], bar(fQFull));
-        for (int j = 0; j < n_kv; ++j, ++gk) {
+        for (int j = j0; j < n_kv; ++j, ++gk) {
           const int st = gk & 1;
           const uint32_t sK = sbase + L::kKV0 + st * L::kStageBytes, sV = sK + L::kTileBytes;
           mbar_wait(bar(fKvEmpty0 + st), ((gk >> 1) & 1) ^ 1, s_abort);
@@ -237,13 +242,14 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         mbar_wait(bar(fUnitFull0 + uc % kFwsUnitRing), (uc / kFwsUnitRing) & 1, s_abort);
         const int u = s_unit[uc % kFwsUnitRing];
         if (u >= n_units || *s_abort) break;
-        const int n_kv = decode_fwd_unit(u, items, order, Hq, G, pair_blocks).n_kv;
+        const FwdUnit w = decode_fwd_unit(u, items, order, Hq, G, pair_blocks, window);
+        const int n_kv = w.n_kv, j0 = w.j0;
         mbar_wait(bar(fQFull), uc & 1, s_abort);
         mbar_wait(bar(fKvFull0 + (gk & 1)), (gk >> 1) & 1, s_abort);
         tc_fence_after();
         issue_s(0, gk & 1);
         issue_s(1, gk & 1);
-        for (int j = 0; j < n_kv; ++j, ++gk) {
+        for (int j = j0; j < n_kv; ++j, ++gk) {
           const int st = gk & 1;
           const uint32_t v_lo =
               desc_lo(sbase + L::kKV0 + st * L::kStageBytes + L::kTileBytes, L::kBoxBytes);
@@ -251,13 +257,13 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
 #pragma unroll
           for (int t = 0; t < 2; ++t) {
             mbar_wait(bar(fPReady0 + t), gk & 1, s_abort);
-            if (j == 0 && uc > 0) mbar_wait(bar(fORead0 + t), (uc - 1) & 1, s_abort);
+            if (j == j0 && uc > 0) mbar_wait(bar(fORead0 + t), (uc - 1) & 1, s_abort);
             tc_fence_after();
             if (leader) {
 #pragma unroll
               for (int kk = 0; kk < kBN / 16; ++kk)   // O_t += P_t V
                 mma_ts(tmem + 256 + t * 128, tmem + t * 128 + kk * 8,
-                       desc_from_lo(v_lo + ((kk * 2048) >> 4)), kIdescPV, (j > 0) | (kk > 0));
+                       desc_from_lo(v_lo + ((kk * 2048) >> 4)), kIdescPV, (j > j0) | (kk > 0));
               if (t == 1) mma_commit(bar(fKvEmpty0 + st));
               if (!more) mma_commit(bar(fOFull0 + t));
             }
@@ -287,23 +293,25 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
       mbar_wait(bar(fUnitFull0 + uc % kFwsUnitRing), (uc / kFwsUnitRing) & 1, s_abort);
       const int u = s_unit[uc % kFwsUnitRing];
       if (u >= n_units || *s_abort) break;
-      const FwdUnit w = decode_fwd_unit(u, items, order, Hq, G, pair_blocks);
+      const FwdUnit w = decode_fwd_unit(u, items, order, Hq, G, pair_blocks, window);
       const int h = w.h[t], q_start = w.q_start[t], q_len = w.q_len[t], diag = w.diag[t];
-      const int n_kv = w.n_kv;
+      const int n_kv = w.n_kv, j0 = w.j0;
       float m_run = -INFINITY, l_run = 0.f;
-      for (int j = 0; j < n_kv; ++j, ++gk) {
+      for (int j = j0; j < n_kv; ++j, ++gk) {
         mbar_wait(bar(fSFull0 + t), gk & 1, s_abort);
         tc_fence_after();
         uint32_t s[128];
 #pragma unroll
         for (int c = 0; c < 4; ++c) tmem_ld32(tS + c * 32, s + c * 32);
         tmem_wait_ld();
-        if (j >= diag) {       // diagonal tile: keys after the query row are masked; a tile past
-                               // the diagonal (block-pair mode, tile 0, last step) entirely
-          const int first_masked = (j == diag) ? row + 1 : 0;
+        // sliding window: keys more than window - 1 before the row are masked too
+        const int lo = (window > 0) ? (q_start + row - (window - 1) - w.kv_start - j * kBN) : 0;
+        if (j >= diag || lo > 0) {   // diagonal tile: keys after the query row are masked; a tile
+                                     // past the diagonal (block-pair mode, tile 0, last step) entirely
+          const int first_masked = (j == diag) ? row + 1 : (j > diag ? 0 : 128);
 #pragma unroll
           for (int c = 0; c < 128; ++c)
-            if (c >= first_masked) s[c] = 0xff800000u;   // -inf
+            if (c >= first_masked || c < lo) s[c] = 0xff800000u;   // -inf
         }
         float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};   // independent chains
 #pragma unroll
@@ -317,16 +325,19 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         const bool changed = row_m > m_run + 8.f;          // true on the first tile (m_run = -inf)
         const float m_new = changed ? row_m : m_run;
         const float alpha = changed ? fast_exp2(m_run - m_new) : 1.f;   // 0 on the first tile
+        // a row that has seen nothing yet (possible only with a sliding window) keeps the maximum
+        // at -inf; the exponentials then use 0 so that they come out as exp2(-inf) = 0, not NaN
+        const float m_sub = (m_new == -INFINITY) ? 0.f : m_new;
         float sum4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
         for (int half = 0; half < 2; ++half) {   // P leaves in two 64-column pieces to bound registers
           uint32_t p[32];
 #pragma unroll
           for (int c = 0; c < 64; c += 4) {
-            const float p0 = fast_exp2(fmaf(__uint_as_float(s[half * 64 + c]), scale_log2, -m_new));
-            const float p1 = fast_exp2(fmaf(__uint_as_float(s[half * 64 + c + 1]), scale_log2, -m_new));
-            const float p2 = fast_exp2(fmaf(__uint_as_float(s[half * 64 + c + 2]), scale_log2, -m_new));
-            const float p3 = fast_exp2(fmaf(__uint_as_float(s[half * 64 + c + 3]), scale_log2, -m_new));
+            const float p0 = fast_exp2(fmaf(__uint_as_float(s[half * 64 + c]), scale_log2, -m_sub));
+            const float p1 = fast_exp2(fmaf(__uint_as_float(s[half * 64 + c + 1]), scale_log2, -m_sub));
+            const float p2 = fast_exp2(fmaf(__uint_as_float(s[half * 64 + c + 2]), scale_log2, -m_sub));
+            const float p3 = fast_exp2(fmaf(__uint_as_float(s[half * 64 + c + 3]), scale_log2, -m_sub));
             sum4[0] += p0; sum4[1] += p1; sum4[2] += p2; sum4[3] += p3;
             p[c >> 1] = pack_bf16x2(p0, p1);
             p[(c >> 1) + 1] = pack_bf16x2(p2, p3);
@@ -336,7 +347,7 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         l_run = l_run * alpha + ((sum4[0] + sum4[1]) + (sum4[2] + sum4[3]));
         m_run = m_new;
         // O_t of step j-1 is complete (its contraction precedes S_t(j) on the tensor pipe)
-        if (j > 0 && __any_sync(0xffffffffu, changed)) {
+        if (j > j0 && __any_sync(0xffffffffu, changed)) {
 #pragma unroll
           for (int c = 0; c < D / 32; ++c) {
             uint32_t o[32];
@@ -381,7 +392,7 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
 template <int D, bool kRot, typename OutT>
 int launch_fws(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, char* ws,
                const WorkspaceLayout& lay, void* out, float* lse, int T, int Hq, int Hkv,
-               float scale, cudaStream_t stream) {
+               float scale, int window, cudaStream_t stream) {
   auto kern = attn_fwd_ws_kernel<D, kRot, OutT>;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            FwsSmem<D>::kTotal) != cudaSuccess)
@@ -394,7 +405,7 @@ int launch_fws(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& 
       tq, tk, tv, reinterpret_cast<const int4*>(ws + lay.off[PK_WS_FWD_ITEMS]),
       reinterpret_cast<const int4*>(ws + lay.off[PK_WS_BWD_ITEMS]),
       reinterpret_cast<const int32_t*>(ws + lay.off[PK_WS_FWD_ORDER]), hdr,
-      static_cast<OutT*>(out), lse, T, Hq, Hkv, scale * kLog2eF);
+      static_cast<OutT*>(out), lse, T, Hq, Hkv, scale * kLog2eF, window);
   return launch_status();
 }
 
@@ -402,9 +413,9 @@ int launch_fws(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& 
 
 int launch_fwd_ws(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, char* ws,
                   const WorkspaceLayout& lay, void* out, float* lse, int T, int Hq, int Hkv, int D,
-                  int out_dtype, float scale, bool rotated, cudaStream_t stream) {
+                  int out_dtype, float scale, int window, bool rotated, cudaStream_t stream) {
 #define PK_FWS(DD, RR, TT) \
-  return launch_fws<DD, RR, TT>(tq, tk, tv, ws, lay, out, lse, T, Hq, Hkv, scale, stream)
+  return launch_fws<DD, RR, TT>(tq, tk, tv, ws, lay, out, lse, T, Hq, Hkv, scale, window, stream)
   if (D == 128) {
     if (rotated) {
       if (out_dtype == PK_BF16) PK_FWS(128, true, __nv_bfloat16); else PK_FWS(128, true, float);

@@ -102,10 +102,10 @@ int plan_launch(const int32_t* position_ids, int32_t T, int32_t* cu_seqlens, int
 int launch_bwd_ws(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
                   const CUtensorMap& tdo, char* ws, const WorkspaceLayout& lay, const float* lse,
                   void* dq, void* dk, void* dv, int T, int Hq, int Hkv, int D, int grad_dtype, float scale,
-                  bool rotated, cudaStream_t stream);
+                  int window, bool rotated, cudaStream_t stream);
 int launch_fwd_ws(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, char* ws,
                   const WorkspaceLayout& lay, void* out, float* lse, int T, int Hq, int Hkv, int D,
-                  int out_dtype, float scale, bool rotated, cudaStream_t stream);
+                  int out_dtype, float scale, int window, bool rotated, cudaStream_t stream);
 // q, k -> rotated fp16 copies (pairs (i, i + D/2), angle pos * theta^(-2i/D))
 int rope_rotate_f16_launch(const void* x, const int32_t* position_ids, int32_t T, int32_t H,
                            int32_t D, float theta, void* y, cudaStream_t stream);

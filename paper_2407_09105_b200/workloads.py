@@ -34,6 +34,7 @@ class Workload:
     rope_theta: float            # <= 0: no rotary embedding
     streams: List[List[int]]     # example lengths of every stream, in stream order
     packing: str                 # which of the paper's packing variants it mimics
+    window: int = 0              # > 0: sliding-window attention, keys visible per row
 
     @property
     def softmax_scale(self) -> float:
@@ -45,8 +46,14 @@ class Workload:
 
     @property
     def causal_pairs(self) -> int:
-        """Sum over examples of L(L+1)/2 (diagonal included)."""
-        return sum(l * (l + 1) // 2 for s in self.streams for l in s)
+        """Sum over examples of L(L+1)/2 (diagonal included); with a sliding window W every
+        row counts min(position + 1, W) keys."""
+        def pairs(l: int) -> int:
+            w = self.window
+            if w <= 0 or l <= w:
+                return l * (l + 1) // 2
+            return w * (w + 1) // 2 + (l - w) * w
+        return sum(pairs(l) for s in self.streams for l in s)
 
     @property
     def useful_flops_fwd(self) -> int:

@@ -20,7 +20,7 @@ def run_plan(pos: torch.Tensor, Hq=1, Hkv=1, D=64):
     return ws, cu, ne, mx
 
 
-def run_fwd(st, w, out_dtype=torch.float32, theta=None, scale=None):
+def run_fwd(st, w, out_dtype=torch.float32, theta=None, scale=None, window=0):
     T, Hq, D = st.q.shape
     Hkv = st.k.shape[1]
     theta = w.rope_theta if theta is None else theta
@@ -28,13 +28,13 @@ def run_fwd(st, w, out_dtype=torch.float32, theta=None, scale=None):
     ws = api.alloc_workspace(T, Hq, Hkv, D)
     out = torch.full((T, Hq, D), float("nan"), dtype=out_dtype, device="cuda")
     lse = torch.full((Hq, T), float("nan"), dtype=torch.float32, device="cuda")
-    api.pk_attn_fwd(st.q, st.k, st.v, st.position_ids, scale, theta, out, lse, ws)
+    api.pk_attn_fwd(st.q, st.k, st.v, st.position_ids, scale, theta, out, lse, ws, window=window)
     code, detail = api.pk_status_read(ws)
     assert code == api.PK_OK, (code, detail)
     return out, lse, ws
 
 
-def run_bwd(st, w, out, lse, ws, grad_dtype=torch.float32, theta=None, scale=None):
+def run_bwd(st, w, out, lse, ws, grad_dtype=torch.float32, theta=None, scale=None, window=0):
     T, Hq, D = st.q.shape
     theta = w.rope_theta if theta is None else theta
     scale = w.softmax_scale if scale is None else scale
@@ -42,7 +42,7 @@ def run_bwd(st, w, out, lse, ws, grad_dtype=torch.float32, theta=None, scale=Non
     dk = torch.full_like(st.k, float("nan"), dtype=grad_dtype)
     dv = torch.full_like(st.v, float("nan"), dtype=grad_dtype)
     api.pk_attn_bwd(st.dout, st.q, st.k, st.v, out, lse, st.position_ids, scale, theta,
-                    dq, dk, dv, ws, reuse_plan=True)
+                    dq, dk, dv, ws, reuse_plan=True, window=window)
     code, detail = api.pk_status_read(ws)
     assert code == api.PK_OK, (code, detail)
     return dq, dk, dv

@@ -50,13 +50,15 @@ def test_argument_validation_returns_codes_without_a_gpu():
     L = api.lib()
     # null workspace / negative T / unsupported shapes are rejected before any CUDA call
     assert L.pk_seqlens_from_posids(None, -1, None, None, None, None, 0, None) == api.PK_ERR_INVALID_ARG
-    assert L.pk_attn_fwd(None, None, None, None, 16, 4, 4, 80, 1.0, 0.0, None, 0, None, 0, None, 0,
+    assert L.pk_attn_fwd(None, None, None, None, 16, 4, 4, 80, 1.0, 0.0, 0, None, 0, None, 0, None, 0,
                          None) == api.PK_ERR_UNSUPPORTED
-    assert L.pk_attn_fwd(None, None, None, None, 16, 4, 4, 64, -1.0, 0.0, None, 0, None, 0, None, 0,
+    assert L.pk_attn_fwd(None, None, None, None, 16, 4, 4, 64, -1.0, 0.0, 0, None, 0, None, 0, None, 0,
                          None) == api.PK_ERR_INVALID_ARG
-    assert L.pk_attn_fwd(None, None, None, None, 16, 4, 4, 64, 1.0, 0.0, None, 7, None, 0, None, 0,
+    assert L.pk_attn_fwd(None, None, None, None, 16, 4, 4, 64, 1.0, 0.0, 0, None, 7, None, 0, None, 0,
                          None) == api.PK_ERR_UNSUPPORTED
-    assert L.pk_attn_bwd(None, None, None, None, None, 0, None, None, 16, 4, 3, 64, 1.0, 0.0, None,
+    assert L.pk_attn_fwd(None, None, None, None, 16, 4, 4, 64, 1.0, 0.0, -1, None, 0, None, 0, None, 0,
+                         None) == api.PK_ERR_INVALID_ARG       # negative window
+    assert L.pk_attn_bwd(None, None, None, None, None, 0, None, None, 16, 4, 3, 64, 1.0, 0.0, 0, None,
                          None, None, 0, 0, None, 0, None) == api.PK_ERR_UNSUPPORTED
     assert L.pk_rope_apply(None, None, 4, 2, 7, 1e4, 0, None) == api.PK_ERR_UNSUPPORTED
     assert L.pk_seqlens_from_posids_noalloc(1, api.PK_NOALLOC_MAX_TOKENS + 1, 1, None, None,
