@@ -16,25 +16,46 @@ __device__ __forceinline__ void red_add_v4(float* addr, float a, float b, float 
                ::"l"(addr), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
 }
 
+// 32 bytes per store where the address allows it: the epilogues write one row per thread, so a
+// warp's store touches 32 different rows, and the load/store unit's time goes with the number
+// of (row, instruction) pairs; full 32-byte sectors also spare L2 the partial writes.
+__device__ __forceinline__ void st_global_v8(void* p, const uint32_t* v) {
+  asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+               ::"l"(p), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]),
+                 "r"(v[6]), "r"(v[7]) : "memory");
+}
+
 template <typename GradT>
 __device__ __forceinline__ void store_chunk32(GradT* dst, const float* x);
 template <>
 __device__ __forceinline__ void store_chunk32<float>(float* dst, const float* x) {
+  if ((reinterpret_cast<uintptr_t>(dst) & 31) == 0) {
+#pragma unroll
+    for (int c = 0; c < 32; c += 8) {
+      uint32_t v[8];
+#pragma unroll
+      for (int e = 0; e < 8; ++e) v[e] = __float_as_uint(x[c + e]);
+      st_global_v8(dst + c, v);
+    }
+    return;
+  }
 #pragma unroll
   for (int c = 0; c < 32; c += 4)
     *reinterpret_cast<float4*>(dst + c) = make_float4(x[c], x[c + 1], x[c + 2], x[c + 3]);
 }
 template <>
 __device__ __forceinline__ void store_chunk32<__nv_bfloat16>(__nv_bfloat16* dst, const float* x) {
+  uint32_t v[16];
 #pragma unroll
-  for (int c = 0; c < 32; c += 8) {
-    uint4 o;
-    o.x = pack_bf16x2(x[c], x[c + 1]);
-    o.y = pack_bf16x2(x[c + 2], x[c + 3]);
-    o.z = pack_bf16x2(x[c + 4], x[c + 5]);
-    o.w = pack_bf16x2(x[c + 6], x[c + 7]);
-    *reinterpret_cast<uint4*>(dst + c) = o;
+  for (int c = 0; c < 16; ++c) v[c] = pack_bf16x2(x[2 * c], x[2 * c + 1]);
+  if ((reinterpret_cast<uintptr_t>(dst) & 31) == 0) {
+    st_global_v8(dst, v);
+    st_global_v8(dst + 16, v + 8);
+    return;
   }
+#pragma unroll
+  for (int c = 0; c < 16; c += 4)
+    *reinterpret_cast<uint4*>(dst + 2 * c) = make_uint4(v[c], v[c + 1], v[c + 2], v[c + 3]);
 }
 
 
