@@ -450,11 +450,16 @@ attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             if (live) {
               const float2* cs = rope_table + (size_t)tok * (D / 2) + c * 32;
 #pragma unroll
-              for (int e = 0; e < 32; ++e) {
-                const float2 t = __ldg(cs + e);
-                const float a = __uint_as_float(x1[e]) * mul, b = __uint_as_float(x2[e]) * mul;
-                y1[e] = a * t.x + b * t.y;
-                y2[e] = b * t.x - a * t.y;
+              for (int e4 = 0; e4 < 32; e4 += 4) {
+                float2 t4[4];
+                ld_table4(cs + e4, t4);
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                  const int e = e4 + k;
+                  const float a = __uint_as_float(x1[e]) * mul, b = __uint_as_float(x2[e]) * mul;
+                  y1[e] = a * t4[k].x + b * t4[k].y;
+                  y2[e] = b * t4[k].x - a * t4[k].y;
+                }
               }
               store_chunk32<GradT>(dst + c * 32, y1);
               store_chunk32<GradT>(dst + D / 2 + c * 32, y2);
@@ -819,11 +824,16 @@ attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
           if (live && mine) {
             const float2* cs = rope_table + (size_t)tok * (D / 2) + qd * 32;
 #pragma unroll
-            for (int e = 0; e < 32; ++e) {
-              const float2 t = __ldg(cs + e);
-              const float a = __uint_as_float(x1[e]) * scale, b = __uint_as_float(x2[e]) * scale;
-              y1[e] = a * t.x + b * t.y;
-              y2[e] = b * t.x - a * t.y;
+            for (int e4 = 0; e4 < 32; e4 += 4) {
+              float2 t4[4];
+              ld_table4(cs + e4, t4);
+#pragma unroll
+              for (int k = 0; k < 4; ++k) {
+                const int e = e4 + k;
+                const float a = __uint_as_float(x1[e]) * scale, b = __uint_as_float(x2[e]) * scale;
+                y1[e] = a * t4[k].x + b * t4[k].y;
+                y2[e] = b * t4[k].x - a * t4[k].y;
+              }
             }
             store_chunk32<GradT>(dst, y1);
             store_chunk32<GradT>(dst + D / 2, y2);
