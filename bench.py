@@ -37,7 +37,7 @@ UNIT = "TFLOP/s"
 
 # DRAM bytes per causal (query, key, q-head) pair of the dominant (dK/dV) kernel, from the ncu
 # capture summarised in profiles/ (scaled to a launch by the number of pairs); None = not captured.
-NCU_BWD_DRAM_BYTES_PER_PAIR = 0.3303   # attn_bwd_dkv_kernel, profiles/attn_kernels_c4_2packs.txt
+NCU_BWD_DRAM_BYTES_PER_PAIR = 0.3330   # attn_bwd_dkv_kernel, profiles/attn_kernels_c4_2packs.txt
 
 
 def _peaks():
