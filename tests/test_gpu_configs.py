@@ -53,7 +53,8 @@ def test_c2_full_flat_stream_fp32():
 
 
 def _sampled(name, n_rows=48, max_example=2600):
-    w = wl.workload(name)
+    w = wl.workload(name) if isinstance(name, str) else name
+    name = w.name
     lens = w.flat_lengths()
     st = wl.stream_tensors(w, lens, 0, device="cuda")
     T, Hq, D = st.q.shape
@@ -113,3 +114,17 @@ def test_c4_sampled_full_size():
 
 def test_c5_sampled_full_size():
     _sampled("c5", n_rows=24, max_example=9000)
+
+
+def test_million_token_stream():
+    # 2^20 tokens in one call (index arithmetic, TMA coordinates and the single-CTA plan at scale):
+    # lengths drawn log-uniformly from 1 .. 40000, two small heads so that memory stays modest
+    rng = np.random.default_rng(77)
+    lens, left = [], 1 << 20
+    while left > 0:
+        n = int(min(left, np.clip(np.rint(np.exp(rng.uniform(0.0, np.log(40000.0)))), 1, 40000)))
+        lens.append(n)
+        left -= n
+    w = wl.Workload("million", 78, 2, 1, 64, 1e4, [lens], "test")
+    assert w.total_tokens == 1 << 20
+    _sampled(w, n_rows=32, max_example=3000)
