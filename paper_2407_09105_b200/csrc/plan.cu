@@ -55,18 +55,31 @@ plan_kernel(const int32_t* __restrict__ pos, int T,
   __syncthreads();
 
   // ---- A: example starts -> cu ------------------------------------------------------
+  // Eight consecutive tokens per thread and round: the loop is bound by the latency of its loads
+  // and barriers, not by their number, so fewer, fatter rounds are what shortens it.
+  constexpr int kPer = 8;
   int carry = 0;
-  for (int base = 0; base < T; base += kPlanThreads) {
-    const int t = base + tid;
-    int flag = 0;
-    if (t < T) {
-      const int p = pos[t];
-      if (p < 0) { set_status(hdr, PK_ERR_BAD_POSIDS, t); s_bad = 1; }
-      flag = (t == 0) || (p <= pos[t - 1]);
+  for (int base = 0; base < T; base += kPlanThreads * kPer) {
+    const int t0 = base + tid * kPer;
+    int p[kPer + 1];
+    p[0] = (t0 > 0 && t0 - 1 < T) ? pos[t0 - 1] : 0;
+#pragma unroll
+    for (int i = 0; i < kPer; ++i) p[i + 1] = (t0 + i < T) ? pos[t0 + i] : 0;
+    unsigned flags = 0;
+#pragma unroll
+    for (int i = 0; i < kPer; ++i) {
+      const int t = t0 + i;
+      if (t < T) {
+        if (p[i + 1] < 0) { set_status(hdr, PK_ERR_BAD_POSIDS, t); s_bad = 1; }
+        if (t == 0 || p[i + 1] <= p[i]) flags |= 1u << i;
+      }
     }
     int tot;
-    const int ex = block_exclusive_scan(flag, &tot, sscan);
-    if (flag) cu[carry + ex] = t;
+    const int ex = block_exclusive_scan(__popc(flags), &tot, sscan);
+    int o = carry + ex;
+#pragma unroll
+    for (int i = 0; i < kPer; ++i)
+      if (flags & (1u << i)) cu[o++] = t0 + i;
     carry += tot;
   }
   const int E = carry;
