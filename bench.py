@@ -290,6 +290,86 @@ def run_loss(args):
     print(json.dumps(line))
 
 
+def run_pack(args):
+    """`--workload pack`: padded batch <-> packed stream for hidden-state rows (4096 bf16 = 8 KB per
+    token) of the first 8 mini-batches of c3 (16 examples each, padded to the longest of the
+    mini-batch), one call per mini-batch and direction.  HBM-bound copies; one JSON line."""
+    from paper_2407_09105_b200 import api
+    from oracle import pad_pack as pp
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
+    w = wl.workload("c3")
+    batches = w.streams[:8]
+    H = 4096
+    gen = torch.Generator(device="cuda").manual_seed(5)
+    items = []
+    for lens in batches:
+        B, lmax, T = len(lens), max(lens), sum(lens)
+        cu = torch.tensor(np.concatenate([[0], np.cumsum(lens)]), dtype=torch.int32, device="cuda")
+        padded = torch.randn((B, lmax, H), generator=gen, device="cuda").to(torch.bfloat16)
+        items.append((cu, padded, torch.empty((T, H), dtype=torch.bfloat16, device="cuda"),
+                      torch.empty_like(padded)))
+    T_all = sum(sum(l) for l in batches)
+    rows_padded = sum(len(l) * max(l) for l in batches)
+    rb = H * 2
+    stream = torch.cuda.current_stream()
+
+    def step_pack():
+        for cu, padded, packed, back in items:
+            api.pk_pack_rows(padded, cu, packed, stream=stream)
+
+    def step_unpack():
+        for cu, padded, packed, back in items:
+            api.pk_unpack_rows(packed, cu, back, stream=stream)
+
+    def timed(fn):
+        for _ in range(max(args.warmup, 3)):
+            fn()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        a.record()
+        for _ in range(args.steps):
+            fn()
+        b.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / args.steps
+
+    ms_pack, ms_unpack = timed(step_pack), timed(step_unpack)
+    peaks = _peaks()
+    pack_bytes = 2.0 * T_all * rb
+    unpack_bytes = (T_all + rows_padded) * float(rb)
+    cpu = None
+    if not args.no_cpu_baseline:
+        cu, padded, packed, back = items[0]
+        x = padded.float().cpu().numpy()
+        t0 = time.perf_counter()
+        y = pp.pack_rows(x, batches[0])
+        pp.unpack_rows(y, batches[0], max(batches[0]))
+        dt = time.perf_counter() - t0
+        cpu = {"value": sum(batches[0]) / dt, "unit": "tokens/s", "cores": 1, "kind": "oracle",
+               "sample": "first mini-batch, pack + unpack in numpy"}
+    ms = ms_pack + ms_unpack
+    line = {
+        "metric": "pad_pack_roundtrip_tokens_per_s", "value": T_all / (ms * 1e-3), "unit": "tokens/s",
+        "n_gpus": 1, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "u8",
+        "data": "synthetic",
+        "config": {"workload": "pack: 8 mini-batches of c3 (16 examples each), 8 KB rows, pack then unpack",
+                   "tokens": T_all, "padded_rows": rows_padded, "row_bytes": rb, "l2": "inputs_exceed_l2"},
+        "e2e": None, "gpu_launches": 2 * len(items) * args.steps,
+        "roofline": {"kernel": "rows_move_kernel<16, unpack>", "bound": "hbm",
+                     "achieved": unpack_bytes / (ms_unpack * 1e-3) / 1e9, "peak": peaks["hbm_gbs"],
+                     "peak_kind": "copy bandwidth, " + peaks["source"], "unit": "GB/s",
+                     "frac": unpack_bytes / (ms_unpack * 1e-3) / 1e9 / peaks["hbm_gbs"], "traffic": None,
+                     "ms_per_step": ms_unpack,
+                     "pack": {"achieved": pack_bytes / (ms_pack * 1e-3) / 1e9,
+                              "frac": pack_bytes / (ms_pack * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                              "ms_per_step": ms_pack}},
+        "cpu_baseline": cpu,
+    }
+    print(json.dumps(line))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -310,6 +390,9 @@ def main():
 
     if args.workload == "loss":
         run_loss(args)
+        return
+    if args.workload == "pack":
+        run_pack(args)
         return
     w = wl.workload(args.workload)
     if args.packs > 0:

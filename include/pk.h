@@ -250,6 +250,22 @@ int pk_pack_next_fit(const int32_t* lengths, int32_t n, int32_t capacity, int32_
                      int32_t* bin_of, int32_t* n_bins);
 
 /*
+ * Between a padded batch and the packed stream (for comparing the two layouts on whole models).
+ * The padded layout is the one the paper starts from (Sec. 3: examples extended to the longest one
+ * with padding appended on the right), the packed one the concatenation of Sec. 3.4.  Rows are
+ * opaque `row_bytes` bytes each (a token id, a hidden vector, ...); device pointers throughout.
+ *   pk_pack_rows     packed[cu[b] + i] = padded[b][i]  for i < cu[b+1] - cu[b]
+ *   pk_unpack_rows   padded[b][i] = packed[cu[b] + i] for those i, zero bytes in the padding rows
+ * padded is [B][l_max][row_bytes], packed [T][row_bytes], cu_seqlens int32 [B+1] with
+ * cu_seqlens[B] = T and every length <= l_max (not checked).  16-byte copies when row_bytes and
+ * both pointers allow it, else 4-byte or single bytes.
+ */
+int pk_pack_rows(const void* padded, const int32_t* cu_seqlens, int32_t B, int32_t l_max, int32_t T,
+                 int64_t row_bytes, void* packed, void* stream);
+int pk_unpack_rows(const void* packed, const int32_t* cu_seqlens, int32_t B, int32_t l_max, int32_t T,
+                   int64_t row_bytes, void* padded, void* stream);
+
+/*
  * Loss of the packed stream (the step right after the model).  The collator's labels carry -100
  * in the first position of every example (Sec. 3.4, worked example in Sec. 3.5); a causal
  * language model scores row t against the label of row t + 1, so with those labels no example

@@ -54,6 +54,8 @@ _SIGNATURES = {
     "pk_collate_padding_free": (ctypes.c_int, [_vp, _vp, _i32, _i32, _vp, _vp, _vp, _i32, _vp]),
     "pk_pack_first_fit_decreasing": (ctypes.c_int, [_vp, _i32, _i32, _vp, ctypes.POINTER(_i32)]),
     "pk_pack_next_fit": (ctypes.c_int, [_vp, _i32, _i32, _i32, _vp, ctypes.POINTER(_i32)]),
+    "pk_pack_rows": (ctypes.c_int, [_vp, _vp, _i32, _i32, _i32, ctypes.c_int64, _vp, _vp]),
+    "pk_unpack_rows": (ctypes.c_int, [_vp, _vp, _i32, _i32, _i32, ctypes.c_int64, _vp, _vp]),
     "pk_packed_loss_fwd": (ctypes.c_int, [_vp, _i32, _vp, _i32, _i32, ctypes.c_int64, _i32, _vp, _vp,
                                           _vp, _vp, _vp]),
     "pk_packed_loss_bwd": (ctypes.c_int, [_vp, _i32, _vp, _vp, _vp, ctypes.c_float, _i32, _i32,
@@ -241,6 +243,31 @@ def pk_collate_padding_free(input_ids: torch.Tensor, lengths: torch.Tensor,
            lib().pk_collate_padding_free(_ptr(input_ids), _ptr(lengths), lengths.numel(),
                                          position_ids.numel(), _ptr(position_ids), _ptr(labels),
                                          _ptr(cu_seqlens), ignore_index, _stream(stream)))
+
+
+def _row_bytes(t: torch.Tensor, lead: int) -> int:
+    n = 1
+    for d in t.shape[lead:]:
+        n *= d
+    return n * t.element_size()
+
+
+def pk_pack_rows(padded: torch.Tensor, cu_seqlens: torch.Tensor, packed: torch.Tensor,
+                 stream=None) -> None:
+    """padded [B, l_max, ...] -> packed [T, ...] (same trailing shape and dtype)."""
+    B, l_max = padded.shape[:2]
+    _check("pk_pack_rows",
+           lib().pk_pack_rows(_ptr(padded), _ptr(cu_seqlens), B, l_max, packed.shape[0],
+                              _row_bytes(packed, 1), _ptr(packed), _stream(stream)))
+
+
+def pk_unpack_rows(packed: torch.Tensor, cu_seqlens: torch.Tensor, padded: torch.Tensor,
+                   stream=None) -> None:
+    """packed [T, ...] -> padded [B, l_max, ...]; padding rows become zero."""
+    B, l_max = padded.shape[:2]
+    _check("pk_unpack_rows",
+           lib().pk_unpack_rows(_ptr(packed), _ptr(cu_seqlens), B, l_max, packed.shape[0],
+                                _row_bytes(packed, 1), _ptr(padded), _stream(stream)))
 
 
 def _logits_dtype(t: torch.Tensor) -> int:

@@ -62,6 +62,69 @@ __global__ void collate_kernel(const int32_t* __restrict__ input_ids, const int3
   if (labels != nullptr) labels[t] = (p == 0) ? ignore_index : input_ids[t];
 }
 
+
+// Padded batch [B][l_max][row_bytes] <-> packed stream [T][row_bytes]; kVec bytes per access.
+// kPack: packed[cu[b] + i] = padded[b][i].  Otherwise the reverse, padding rows zero-filled.
+// One CTA per destination row (blockIdx.x) and slice of it (blockIdx.y): the row's source is
+// looked up once per CTA, and the threads stream the bytes without any index arithmetic.
+template <int kVec, bool kPack>
+__global__ void __launch_bounds__(256)
+rows_move_kernel(const uint8_t* __restrict__ src, const int32_t* __restrict__ cu, int B, int l_max,
+                 long long row_bytes, uint8_t* __restrict__ dst) {
+  const long long r = blockIdx.x;
+  long long from;
+  bool copy = true;
+  if (kPack) {
+    int lo = 0, hi = B - 1;                 // largest b with cu[b] <= r (uniform for the CTA)
+    while (lo < hi) {
+      const int mid = (lo + hi + 1) >> 1;
+      if (cu[mid] <= r) lo = mid; else hi = mid - 1;
+    }
+    from = (long long)lo * l_max + (r - cu[lo]);
+  } else {
+    const int b = (int)(r / l_max), i = (int)(r % l_max);
+    copy = i < cu[b + 1] - cu[b];
+    from = (long long)cu[b] + i;
+  }
+  const uint8_t* s = src + from * row_bytes;
+  uint8_t* d = dst + r * row_bytes;
+  const long long chunks = row_bytes / kVec;
+  constexpr int kPerThread = 4;
+  const long long c0 = ((long long)blockIdx.y * kPerThread) * 256 + threadIdx.x;
+#pragma unroll
+  for (int k = 0; k < kPerThread; ++k) {
+    const long long c = c0 + (long long)k * 256;
+    if (c >= chunks) break;
+    if (kVec == 16) {
+      reinterpret_cast<uint4*>(d)[c] = copy ? reinterpret_cast<const uint4*>(s)[c] : make_uint4(0, 0, 0, 0);
+    } else if (kVec == 4) {
+      reinterpret_cast<uint32_t*>(d)[c] = copy ? reinterpret_cast<const uint32_t*>(s)[c] : 0u;
+    } else {
+      d[c] = copy ? s[c] : (uint8_t)0;
+    }
+  }
+}
+
+template <bool kPack>
+int rows_move(const void* src, const int32_t* cu, int B, int l_max, int T, long long row_bytes,
+              void* dst, cudaStream_t stream) {
+  const long long n_rows = kPack ? (long long)T : (long long)B * l_max;
+  if (n_rows == 0) return PK_OK;
+  if (n_rows > 0x7fffffffLL) return PK_ERR_UNSUPPORTED;
+  const uintptr_t a = reinterpret_cast<uintptr_t>(src) | reinterpret_cast<uintptr_t>(dst) |
+                      (uintptr_t)row_bytes;
+  const int vec = (a & 15) == 0 ? 16 : ((a & 3) == 0 ? 4 : 1);
+  const long long slices = (row_bytes / vec + 4 * 256 - 1) / (4 * 256);
+  if (slices > 65535) return PK_ERR_UNSUPPORTED;
+  const dim3 grid((unsigned)n_rows, (unsigned)slices);
+  const auto* s = static_cast<const uint8_t*>(src);
+  auto* d = static_cast<uint8_t*>(dst);
+  if (vec == 16) rows_move_kernel<16, kPack><<<grid, 256, 0, stream>>>(s, cu, B, l_max, row_bytes, d);
+  else if (vec == 4) rows_move_kernel<4, kPack><<<grid, 256, 0, stream>>>(s, cu, B, l_max, row_bytes, d);
+  else rows_move_kernel<1, kPack><<<grid, 256, 0, stream>>>(s, cu, B, l_max, row_bytes, d);
+  return launch_status();
+}
+
 }  // namespace
 }  // namespace pk
 
@@ -123,4 +186,21 @@ extern "C" int pk_pack_next_fit(const int32_t* lengths, int32_t n, int32_t capac
   }
   *n_bins = started ? b + 1 : 0;
   return PK_OK;
+}
+
+extern "C" int pk_pack_rows(const void* padded, const int32_t* cu_seqlens, int32_t B, int32_t l_max,
+                            int32_t T, int64_t row_bytes, void* packed, void* stream) {
+  if (B < 0 || l_max < 0 || T < 0 || row_bytes <= 0) return PK_ERR_INVALID_ARG;
+  if (T > 0 && (!padded || !packed || !cu_seqlens || B == 0)) return PK_ERR_INVALID_ARG;
+  return pk::rows_move<true>(padded, cu_seqlens, B, l_max, T, row_bytes, packed,
+                             static_cast<cudaStream_t>(stream));
+}
+
+extern "C" int pk_unpack_rows(const void* packed, const int32_t* cu_seqlens, int32_t B, int32_t l_max,
+                              int32_t T, int64_t row_bytes, void* padded, void* stream) {
+  if (B < 0 || l_max < 0 || T < 0 || row_bytes <= 0) return PK_ERR_INVALID_ARG;
+  if ((long long)B * l_max > 0 && (!padded || !cu_seqlens || (T > 0 && !packed)))
+    return PK_ERR_INVALID_ARG;
+  return pk::rows_move<false>(packed, cu_seqlens, B, l_max, T, row_bytes, padded,
+                              static_cast<cudaStream_t>(stream));
 }

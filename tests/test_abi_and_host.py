@@ -74,6 +74,12 @@ def test_argument_validation_returns_codes_without_a_gpu():
     assert L.pk_packed_loss_fwd(None, 0, None, 4, 8, 8, -100, None, None, 1, 1, None) == bad     # no logits
     assert L.pk_packed_loss_bwd(None, 0, None, None, None, 1.0, 4, 8, 8, -100, None, None) == bad
     assert L.pk_packed_loss_bwd(None, 0, None, None, 1, 1.0, 0, 8, 8, -100, None, None) == api.PK_OK  # T = 0
+    # padded <-> packed
+    assert L.pk_pack_rows(None, None, 2, 4, 6, 0, None, None) == bad          # row_bytes
+    assert L.pk_pack_rows(None, None, 2, 4, 6, 8, None, None) == bad          # null buffers
+    assert L.pk_pack_rows(None, None, 2, 4, 0, 8, None, None) == api.PK_OK    # nothing to move
+    assert L.pk_unpack_rows(None, None, -1, 4, 0, 8, None, None) == bad
+    assert L.pk_unpack_rows(None, None, 0, 4, 0, 8, None, None) == api.PK_OK
 
 
 def test_assign_streams_balances_by_pairs():
