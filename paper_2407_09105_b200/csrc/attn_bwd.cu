@@ -517,8 +517,9 @@ extern "C" int pk_attn_bwd(const void* dout, const void* q, const void* k, const
   const bool use_rope = rope_theta > 0.f;
   const bool rotated_copies = use_rope && g_rope_mode == PK_ROPE_ROTATED_COPIES;
   float* table = reinterpret_cast<float*>(ws + lay.off[PK_WS_ROPE_TABLE]);
-  if (use_rope) {
-    rc = rope_table_launch(position_ids, T, D, rope_theta, table, stream);
+  if (use_rope) {   // reduced angles for the warp-specialised kernels' epilogues, (cos, sin) in-tile
+    rc = rotated_copies ? rope_angle_launch(position_ids, T, D, rope_theta, table, stream)
+                        : rope_table_launch(position_ids, T, D, rope_theta, table, stream);
     if (rc != PK_OK) return rc;
   }
   float* delta = reinterpret_cast<float*>(ws + lay.off[PK_WS_DELTA]);

@@ -98,7 +98,7 @@ attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     const int4* __restrict__ items, const int32_t* __restrict__ order, int32_t* hdr,
                     const float* __restrict__ lse, const float* __restrict__ delta,
                     GradT* __restrict__ dk, GradT* __restrict__ dv,
-                    const float2* __restrict__ rope_table,
+                    const float* __restrict__ rope_angle,
                     int T, int Hq, int Hkv, float scale, float scale_log2, int window) {
   using L = DkvSmem<D>;
   extern __shared__ __align__(1024) uint8_t smem[];
@@ -448,13 +448,13 @@ attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             tmem_ld32(src + D / 2 + c * 32, x2);
             tmem_wait_ld();
             if (live) {
-              const float2* cs = rope_table + (size_t)tok * (D / 2) + c * 32;
+              const float* cs = rope_angle + (size_t)tok * (D / 2) + c * 32;
 #pragma unroll
-              for (int e4 = 0; e4 < 32; e4 += 4) {
-                float2 t4[4];
-                ld_table4(cs + e4, t4);
+              for (int e4 = 0; e4 < 32; e4 += 8) {
+                float2 t4[8];
+                ld_angles8(cs + e4, t4);
 #pragma unroll
-                for (int k = 0; k < 4; ++k) {
+                for (int k = 0; k < 8; ++k) {
                   const int e = e4 + k;
                   const float a = __uint_as_float(x1[e]) * mul, b = __uint_as_float(x2[e]) * mul;
                   y1[e] = a * t4[k].x + b * t4[k].y;
@@ -526,7 +526,7 @@ attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                    const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_do,
                    const int4* __restrict__ items, const int32_t* __restrict__ order, int32_t* hdr,
                    const float* __restrict__ lse, const float* __restrict__ delta,
-                   GradT* __restrict__ dq, const float2* __restrict__ rope_table, int T, int Hq,
+                   GradT* __restrict__ dq, const float* __restrict__ rope_angle, int T, int Hq,
                    int Hkv, float scale, float scale_log2, int window) {
   using L = DqSmem<D>;
   extern __shared__ __align__(1024) uint8_t smem[];
@@ -822,13 +822,13 @@ attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
           }
           tmem_wait_ld();
           if (live && mine) {
-            const float2* cs = rope_table + (size_t)tok * (D / 2) + qd * 32;
+            const float* cs = rope_angle + (size_t)tok * (D / 2) + qd * 32;
 #pragma unroll
-            for (int e4 = 0; e4 < 32; e4 += 4) {
-              float2 t4[4];
-              ld_table4(cs + e4, t4);
+            for (int e4 = 0; e4 < 32; e4 += 8) {
+              float2 t4[8];
+              ld_angles8(cs + e4, t4);
 #pragma unroll
-              for (int k = 0; k < 4; ++k) {
+              for (int k = 0; k < 8; ++k) {
                 const int e = e4 + k;
                 const float a = __uint_as_float(x1[e]) * scale, b = __uint_as_float(x2[e]) * scale;
                 y1[e] = a * t4[k].x + b * t4[k].y;
@@ -877,7 +877,7 @@ int launch_ws(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& t
     return PK_ERR_CUDA;
   int32_t* hdr = reinterpret_cast<int32_t*>(ws + lay.off[PK_WS_HEADER]);
   const float* delta = reinterpret_cast<const float*>(ws + lay.off[PK_WS_DELTA]);
-  const float2* table = reinterpret_cast<const float2*>(ws + lay.off[PK_WS_ROPE_TABLE]);
+  const float* table = reinterpret_cast<const float*>(ws + lay.off[PK_WS_ROPE_TABLE]);   // reduced angles
   const int grid = sm_count();
   // the two unit counters (adjacent header slots) start every call at zero
   static_assert(kHdrDqTicket == kHdrBwdTicket + 1, "one memset covers both counters");

@@ -25,15 +25,17 @@ __device__ __forceinline__ void st_global_v8(void* p, const uint32_t* v) {
                  "r"(v[6]), "r"(v[7]) : "memory");
 }
 
-// four (cos, sin) pairs of the rotation table per load (rows of the table are 32-byte aligned)
-__device__ __forceinline__ void ld_table4(const float2* p, float2* t) {
+// eight reduced rotation angles per load (rows of the angle table are 32-byte aligned), turned
+// into (cos, sin) with the fast intrinsics: the angles lie in [-pi, pi], where those are accurate
+// to 4e-7
+__device__ __forceinline__ void ld_angles8(const float* p, float2* t) {
   float v[8];
   asm volatile("ld.global.nc.v8.f32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
                : "=f"(v[0]), "=f"(v[1]), "=f"(v[2]), "=f"(v[3]), "=f"(v[4]), "=f"(v[5]), "=f"(v[6]),
                  "=f"(v[7])
                : "l"(p));
 #pragma unroll
-  for (int e = 0; e < 4; ++e) t[e] = make_float2(v[2 * e], v[2 * e + 1]);
+  for (int e = 0; e < 8; ++e) __sincosf(v[e], &t[e].y, &t[e].x);
 }
 
 template <typename GradT>

@@ -106,6 +106,9 @@ int launch_bwd_ws(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMa
 int launch_fwd_ws(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, char* ws,
                   const WorkspaceLayout& lay, void* out, float* lse, int T, int Hq, int Hkv, int D,
                   int out_dtype, float scale, int window, bool rotated, cudaStream_t stream);
+// reduced angles [T][D/2] fp32 for the epilogues of the rotated-copies path
+int rope_angle_launch(const int32_t* position_ids, int32_t T, int32_t D, float theta, float* angle,
+                      cudaStream_t stream);
 // q, k -> rotated fp16 copies (pairs (i, i + D/2), angle pos * theta^(-2i/D))
 int rope_rotate_f16_launch(const void* x, const int32_t* position_ids, int32_t T, int32_t H,
                            int32_t D, float theta, void* y, cudaStream_t stream);

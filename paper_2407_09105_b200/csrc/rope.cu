@@ -32,6 +32,21 @@ __global__ void rope_table_kernel(const int32_t* __restrict__ pos, int T, int D,
   table[idx] = make_float2(c, s);
 }
 
+// angle[t][i] = pos[t] * theta^(-2i/D) reduced to [-pi, pi] (in fp64, then rounded to fp32): what the
+// epilogues of the rotated-copies path read.  Half the bytes of a (cos, sin) pair per entry, which
+// is what their row-per-thread loads are bound by; they take sine and cosine with the fast
+// intrinsics, accurate to 4e-7 on that range.
+__global__ void rope_angle_kernel(const int32_t* __restrict__ pos, int T, int D, double log2_theta,
+                                  float* __restrict__ angle) {
+  const int half = D / 2;
+  const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= (int64_t)T * half) return;
+  const int t = (int)(idx / half), i = (int)(idx % half);
+  const double a = (double)pos[t] * exp2(-2.0 * (double)i / (double)D * log2_theta);
+  const double two_pi = 6.283185307179586476925286766559;
+  angle[idx] = (float)(a - two_pi * rint(a / two_pi));
+}
+
 // One thread per (token, pair index); loops over heads so cos/sin are formed once.
 __global__ void rope_apply_kernel(__nv_bfloat16* __restrict__ x, const int32_t* __restrict__ pos,
                                   int T, int H, int D, double log2_theta, int inverse) {
@@ -118,6 +133,16 @@ int rope_rotate_f16_launch(const void* x, const int32_t* position_ids, int32_t T
   rope_rotate_f16_kernel<<<blocks, threads, 0, stream>>>(
       static_cast<const __nv_bfloat16*>(x), position_ids, T, H, D, log2((double)theta),
       static_cast<__half*>(y));
+  return launch_status();
+}
+
+int rope_angle_launch(const int32_t* position_ids, int32_t T, int32_t D, float theta,
+                      float* angle, cudaStream_t stream) {
+  if (T == 0) return PK_OK;
+  const int64_t n = (int64_t)T * (D / 2);
+  const int threads = 256;
+  const unsigned blocks = (unsigned)((n + threads - 1) / threads);
+  rope_angle_kernel<<<blocks, threads, 0, stream>>>(position_ids, T, D, log2((double)theta), angle);
   return launch_status();
 }
 
