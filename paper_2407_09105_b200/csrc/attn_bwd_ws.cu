@@ -1,4 +1,5 @@
-// Warp-specialised backward kernels (no fused RoPE) for sm_100a.
+// Warp-specialised backward kernels for sm_100a (with RoPE they run on rotated fp16 copies of q
+// and k and rotate dQ / dK back in their epilogues: kRot).
 //
 // The backward is split into two kernels so that no gradient needs floating-point atomics
 // (fp32 reductions into a dQ accumulator ran at about 2 TB/s here and took longer than all
@@ -13,7 +14,8 @@
 //         S = Q K^T, dP = dO V^T, dS = P o (dP - delta), dQ += dS K   (dQ stays in tensor memory)
 //
 // Both recompute S and dP (7 contractions per tile pair instead of 5), both are bitwise
-// reproducible, and both never visit a tile outside an example's causal block.
+// reproducible, and both never visit a tile outside an example's causal block (or, with a
+// sliding window, outside the band of tiles the window reaches).
 //
 // Roles: 8 compute warps (lane = tensor-memory row; warp w works on columns [64*(w/4), +64) of
 // the rows of lane quarter w%4; 16 warps of 32 columns measured slightly slower because they
@@ -36,7 +38,7 @@ using namespace ptx;
 #ifndef PK_BWD_COMPUTE_THREADS
 #define PK_BWD_COMPUTE_THREADS 256
 #endif
-constexpr int kComputeThreads = PK_BWD_COMPUTE_THREADS;   // 256 or 512
+constexpr int kComputeThreads = PK_BWD_COMPUTE_THREADS;
 constexpr int kNQ = kComputeThreads / 128;                // column groups per tile row
 constexpr int kCW = 128 / kNQ;                            // columns per compute thread
 constexpr int kWsThreads = kComputeThreads + 64;
@@ -54,7 +56,6 @@ constexpr float kLog2eWs = 1.4426950408889634f;
 // later; no role can fall that far behind the TMA warp, which waits for the previous unit's
 // tiles to be released before it loads the next one's.
 constexpr int kUnitRing = 4;
-
 
 // =========================================================================================
 // dK / dV kernel
