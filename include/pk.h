@@ -235,6 +235,20 @@ int pk_collate_padding_free(const int32_t* input_ids, const int32_t* lengths, in
                             int32_t ignore_index, void* stream);
 
 /*
+ * Fixed-length packing with position ids (Sec. 3.3 and Table 1: the packing variant that uses
+ * position ids but still breaks examples): as pk_collate_padding_free, and in addition the stream
+ * is cut into packs of msl tokens (pack k = tokens [k*msl, (k+1)*msl); the last one may be
+ * short).  The paper does not describe the ids of the tail of a broken example; here a pack is a
+ * sequence of its own, so the fragment that opens a pack is a new example: its position ids
+ * restart at 0 and its first label becomes ignore_index.  cu_seqlens still receives the prefix
+ * sums of the given lengths ([E+1]); the boundaries the attention calls use are the ones they
+ * recover from position_ids (example starts and pack starts).  msl <= 0 is PK_ERR_INVALID_ARG.
+ */
+int pk_collate_fixed_length(const int32_t* input_ids, const int32_t* lengths, int32_t E, int32_t T,
+                            int32_t msl, int32_t* position_ids, int32_t* labels,
+                            int32_t* cu_seqlens, int32_t ignore_index, void* stream);
+
+/*
  * Sample selection (Sec. 3.3), on the HOST (all pointers are host pointers): bin_of[i] receives
  * the pack of example i, *n_bins the number of packs.  Every length must be in [1, capacity].
  *   first_fit_decreasing  Multipack-style: examples from long to short (ties in the given

@@ -52,6 +52,7 @@ _SIGNATURES = {
     "pk_set_timing_events": (ctypes.c_int, [_i32, _vp, _vp]),
     "pk_set_rope_mode": (ctypes.c_int, [_i32]),
     "pk_collate_padding_free": (ctypes.c_int, [_vp, _vp, _i32, _i32, _vp, _vp, _vp, _i32, _vp]),
+    "pk_collate_fixed_length": (ctypes.c_int, [_vp, _vp, _i32, _i32, _i32, _vp, _vp, _vp, _i32, _vp]),
     "pk_pack_first_fit_decreasing": (ctypes.c_int, [_vp, _i32, _i32, _vp, ctypes.POINTER(_i32)]),
     "pk_pack_next_fit": (ctypes.c_int, [_vp, _i32, _i32, _i32, _vp, ctypes.POINTER(_i32)]),
     "pk_pack_rows": (ctypes.c_int, [_vp, _vp, _i32, _i32, _i32, ctypes.c_int64, _vp, _vp]),
@@ -243,6 +244,16 @@ def pk_collate_padding_free(input_ids: torch.Tensor, lengths: torch.Tensor,
            lib().pk_collate_padding_free(_ptr(input_ids), _ptr(lengths), lengths.numel(),
                                          position_ids.numel(), _ptr(position_ids), _ptr(labels),
                                          _ptr(cu_seqlens), ignore_index, _stream(stream)))
+
+
+def pk_collate_fixed_length(input_ids: torch.Tensor, lengths: torch.Tensor, msl: int,
+                            position_ids: torch.Tensor, labels: Optional[torch.Tensor],
+                            cu_seqlens: torch.Tensor, ignore_index: int = -100, stream=None) -> None:
+    _check("pk_collate_fixed_length",
+           lib().pk_collate_fixed_length(_ptr(input_ids), _ptr(lengths), lengths.numel(),
+                                         position_ids.numel(), msl, _ptr(position_ids),
+                                         _ptr(labels), _ptr(cu_seqlens), ignore_index,
+                                         _stream(stream)))
 
 
 def _row_bytes(t: torch.Tensor, lead: int) -> int:

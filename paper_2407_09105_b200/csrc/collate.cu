@@ -1,5 +1,6 @@
 // Steps around the attention path ("next" scope): the padding-free collator of Sec. 3.4 / 3.5 on
-// the device (position ids restart per example, first label of an example is ignored), and the
+// the device (position ids restart per example, first label of an example is ignored), its
+// fixed-length variant (the stream cut into packs of msl tokens, Sec. 3.3), and the
 // sample-selection baselines of Sec. 3.3 on the host (first-fit-decreasing as in Multipack, and
 // first-come-first-served filling).
 #include <algorithm>
@@ -47,9 +48,11 @@ __global__ void __launch_bounds__(1024) lengths_scan_kernel(const int32_t* __res
   }
 }
 
+// msl > 0: the stream is also cut at every multiple of msl (fixed-length packing, Sec. 3.3): the
+// fragment that opens a pack counts as a new example.
 __global__ void collate_kernel(const int32_t* __restrict__ input_ids, const int32_t* __restrict__ cu,
-                               int E, int T, int32_t ignore_index, int32_t* __restrict__ position_ids,
-                               int32_t* __restrict__ labels) {
+                               int E, int T, int msl, int32_t ignore_index,
+                               int32_t* __restrict__ position_ids, int32_t* __restrict__ labels) {
   const int t = blockIdx.x * blockDim.x + threadIdx.x;
   if (t >= T) return;
   int lo = 0, hi = E - 1;                 // largest e with cu[e] <= t
@@ -57,7 +60,9 @@ __global__ void collate_kernel(const int32_t* __restrict__ input_ids, const int3
     const int mid = (lo + hi + 1) >> 1;
     if (cu[mid] <= t) lo = mid; else hi = mid - 1;
   }
-  const int p = t - cu[lo];
+  int start = cu[lo];
+  if (msl > 0) start = max(start, t - t % msl);
+  const int p = t - start;
   position_ids[t] = p;
   if (labels != nullptr) labels[t] = (p == 0) ? ignore_index : input_ids[t];
 }
@@ -128,9 +133,11 @@ int rows_move(const void* src, const int32_t* cu, int B, int l_max, int T, long 
 }  // namespace
 }  // namespace pk
 
-extern "C" int pk_collate_padding_free(const int32_t* input_ids, const int32_t* lengths, int32_t E,
-                                       int32_t T, int32_t* position_ids, int32_t* labels,
-                                       int32_t* cu_seqlens, int32_t ignore_index, void* stream_) {
+namespace pk {
+namespace {
+int collate(const int32_t* input_ids, const int32_t* lengths, int32_t E, int32_t T, int32_t msl,
+            int32_t* position_ids, int32_t* labels, int32_t* cu_seqlens, int32_t ignore_index,
+            void* stream_) {
   if (E < 0 || T < 0 || cu_seqlens == nullptr) return PK_ERR_INVALID_ARG;
   if ((E > 0 && lengths == nullptr) || (T > 0 && position_ids == nullptr)) return PK_ERR_INVALID_ARG;
   if (T > 0 && (E == 0 || (labels != nullptr && input_ids == nullptr))) return PK_ERR_INVALID_ARG;
@@ -138,9 +145,27 @@ extern "C" int pk_collate_padding_free(const int32_t* input_ids, const int32_t* 
   pk::lengths_scan_kernel<<<1, 1024, 0, stream>>>(lengths, E, cu_seqlens);
   if (pk::launch_status() != PK_OK) return PK_ERR_CUDA;
   if (T == 0) return PK_OK;
-  pk::collate_kernel<<<(T + 255) / 256, 256, 0, stream>>>(input_ids, cu_seqlens, E, T, ignore_index,
-                                                         position_ids, labels);
+  pk::collate_kernel<<<(T + 255) / 256, 256, 0, stream>>>(input_ids, cu_seqlens, E, T, msl,
+                                                         ignore_index, position_ids, labels);
   return pk::launch_status();
+}
+}  // namespace
+}  // namespace pk
+
+extern "C" int pk_collate_padding_free(const int32_t* input_ids, const int32_t* lengths, int32_t E,
+                                       int32_t T, int32_t* position_ids, int32_t* labels,
+                                       int32_t* cu_seqlens, int32_t ignore_index, void* stream) {
+  return pk::collate(input_ids, lengths, E, T, 0, position_ids, labels, cu_seqlens, ignore_index,
+                     stream);
+}
+
+extern "C" int pk_collate_fixed_length(const int32_t* input_ids, const int32_t* lengths, int32_t E,
+                                       int32_t T, int32_t msl, int32_t* position_ids,
+                                       int32_t* labels, int32_t* cu_seqlens, int32_t ignore_index,
+                                       void* stream) {
+  if (msl <= 0) return PK_ERR_INVALID_ARG;
+  return pk::collate(input_ids, lengths, E, T, msl, position_ids, labels, cu_seqlens, ignore_index,
+                     stream);
 }
 
 extern "C" int pk_pack_first_fit_decreasing(const int32_t* lengths, int32_t n, int32_t capacity,

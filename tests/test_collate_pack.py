@@ -39,6 +39,54 @@ def test_collator_reproduces_the_papers_example():
     assert cu2[:E + 1].tolist() == cu
 
 
+def test_fixed_length_collator_pins():
+    g = _golden()
+    T = len(g["input_ids"])
+    # a pack at least as long as the stream cuts nothing: the paper's worked example again
+    for msl in (T, T + 1, 1000):
+        ids, labels, pos, starts = orc.collate_fixed_length(EXAMPLES, msl)
+        assert ids == g["input_ids"] and labels == g["labels"] and pos == g["position_ids"]
+        assert starts == g["cu_seqlens"]
+    # hand-worked: lengths 4, 8, 5, 11 cut every 10 tokens -> boundaries at the example starts
+    # 0 4 12 17 and at the pack starts 10 20
+    ids, labels, pos, starts = orc.collate_fixed_length(EXAMPLES, 10)
+    assert starts == [0, 4, 10, 12, 17, 20, 28]
+    assert pos == [0, 1, 2, 3, 0, 1, 2, 3, 4, 5, 0, 1, 0, 1, 2, 3, 4, 0, 1, 2, 0, 1, 2, 3, 4, 5, 6, 7]
+    assert [t for t, l in enumerate(labels) if l == -100] == starts[:-1]
+    assert all(l == i for l, i in zip(labels, ids) if l != -100) and ids == g["input_ids"]
+    # every pack taken alone is a well-formed padding-free stream: it equals the padding-free
+    # collation of the pieces that fall into it (random lengths, several pack sizes)
+    rng = np.random.default_rng(11)
+    for msl in (1, 7, 64):
+        examples = [list(rng.integers(0, 1000, size=n)) for n in rng.integers(1, 40, size=30)]
+        ids, labels, pos, starts = orc.collate_fixed_length(examples, msl)
+        flat = [t for e in examples for t in e]
+        ex_of = [i for i, e in enumerate(examples) for _ in e]
+        for k in range(0, len(flat), msl):
+            piece_ids = flat[k:k + msl]
+            pieces = [[t for t, _ in grp] for _, grp in
+                      itertools.groupby(zip(piece_ids, ex_of[k:k + msl]), key=lambda x: x[1])]
+            i2, l2, p2, _ = orc.collate_padding_free(pieces)
+            assert ids[k:k + msl] == i2 and labels[k:k + msl] == l2 and pos[k:k + msl] == p2
+        # and the boundary recovery of the attention path finds exactly these fragments
+        cu2, E, _ = orc_attn.seqlens_from_posids(pos)
+        assert cu2[:E + 1].tolist() == starts
+
+
+def test_fixed_length_collator_gives_the_fragments_of_the_fixed_length_workload():
+    # the c2 generator cuts its drawn lengths into fragments per pack; the collator's boundaries
+    # on the same lengths must be those fragments
+    from paper_2407_09105_b200 import workloads as wl
+    w = wl.workload("c2")
+    frags = [l for pack in w.streams for l in pack]
+    # undo the cuts: a fragment that starts at a multiple of 4096 may continue an example, which the
+    # generator does not record, so feed the fragments themselves (cutting is idempotent)
+    examples = [[0] * l for l in frags]
+    _, _, pos, starts = orc.collate_fixed_length(examples, 4096)
+    assert np.diff(starts).tolist() == frags
+    assert pos == wl.position_ids_from_lengths(frags).tolist()
+
+
 def _optimal_bins(lengths, cap):
     """Brute force: smallest number of bins over all assignments (tiny inputs only)."""
     n = len(lengths)
@@ -120,6 +168,35 @@ def test_device_collator_matches_the_papers_example_and_the_oracle():
         d_cu = torch.full((len(examples) + 1,), -7, dtype=torch.int32, device="cuda")
         api.pk_collate_padding_free(d_ids, d_len, d_pos, d_lab, d_cu)
         assert d_pos.tolist() == pos and d_lab.tolist() == labels and d_cu.tolist() == cu
+
+
+@pytest.mark.gpu
+def test_device_fixed_length_collator_matches_the_oracle():
+    rng = np.random.default_rng(5)
+    cases = [(EXAMPLES, 10), (EXAMPLES, 28), (EXAMPLES, 1), ([[7]], 4),
+             ([list(range(1, 3001)), [5], list(range(9))], 256),
+             ([list(rng.integers(0, 9999, size=n)) for n in rng.integers(1, 900, size=400)], 4096)]
+    for examples, msl in cases:
+        ids, labels, pos, starts = orc.collate_fixed_length(examples, msl)
+        lens = [len(e) for e in examples]
+        d_ids = torch.tensor(ids, dtype=torch.int32, device="cuda")
+        d_len = torch.tensor(lens, dtype=torch.int32, device="cuda")
+        d_pos = torch.full_like(d_ids, -7)
+        d_lab = torch.full_like(d_ids, -7)
+        d_cu = torch.full((len(examples) + 1,), -7, dtype=torch.int32, device="cuda")
+        api.pk_collate_fixed_length(d_ids, d_len, msl, d_pos, d_lab, d_cu)
+        assert d_pos.tolist() == pos and d_lab.tolist() == labels
+        assert d_cu.tolist() == [0] + list(np.cumsum(lens))
+        # the attention path's scan recovers the fragments
+        T = len(ids)
+        ws = api.alloc_workspace(T, 1, 1, 64)
+        cu2 = torch.empty((T + 1,), dtype=torch.int32, device="cuda")
+        ne = torch.empty((1,), dtype=torch.int32, device="cuda")
+        mx = torch.empty((1,), dtype=torch.int32, device="cuda")
+        api.pk_seqlens_from_posids(d_pos, cu2, ne, mx, ws)
+        assert cu2[:int(ne) + 1].tolist() == starts
+    with pytest.raises(api.PkError):
+        api.pk_collate_fixed_length(d_ids, d_len, 0, d_pos, d_lab, d_cu)
 
 
 @pytest.mark.gpu
