@@ -1,11 +1,17 @@
-// Backward of packed (block-diagonal causal) attention on sm_100a.
+// Backward of packed (block-diagonal causal) attention on sm_100a: the entry point pk_attn_bwd
+// (bottom of the file), the row-sum pre-pass delta = sum_d dO*O, and the single-kernel backward
+// with RoPE applied inside the tile.
 //
-// Three launches: (1) the row-sum pre-pass delta = sum_d dO*O, (2) the main kernel, which is
-// key-tile stationary: one unit = (a block of <= 128 key rows of one example, one kv head); it
+// pk_attn_bwd plans (or reuses the plan), runs the pre-pass and then the two warp-specialised
+// kernels of attn_bwd_ws.cu (dK/dV, then dQ; no reductions through memory): directly on q and k
+// without RoPE, on rotated fp16 copies with it (the default RoPE mode).  Only the in-tile RoPE
+// mode (pk_set_rope_mode) runs the main kernel of this file:
+//
+// It is key-tile stationary: one unit = (a block of <= 128 key rows of one example, one kv head); it
 // walks the query tiles from the diagonal to the end of the example for each of the G query
 // heads of the group, keeps dK and dV in tensor memory for the whole unit (fixed accumulation
 // order, so their rows are bitwise reproducible) and sends each query tile's dQ contribution
-// to an fp32 accumulator with vector reductions, (3) a pass that scales, un-rotates and casts
+// to an fp32 accumulator with vector reductions; a last pass scales, un-rotates and casts
 // dQ.  Query tiles outside the example are never visited (Table 1, "Correct Cross-Attention").
 //
 // Per step, with the key rows on the tensor-memory lanes:

@@ -1,4 +1,9 @@
-// Forward of packed (block-diagonal causal) attention on sm_100a.
+// Forward of packed (block-diagonal causal) attention on sm_100a: the entry point pk_attn_fwd
+// (bottom of the file) and the single-tile kernel with RoPE applied inside the tile.
+//
+// pk_attn_fwd plans (or reuses the plan), then runs the warp-specialised two-tile kernel of
+// attn_fwd_ws.cu: directly on q and k without RoPE, on rotated fp16 copies with it (the default
+// RoPE mode).  Only the in-tile RoPE mode (pk_set_rope_mode) runs the kernel of this file:
 //
 // Work comes from the plan's forward list: one unit = (a block of <= 128 query rows of one
 // example, one query head).  Only the key tiles between the example start and the block's
@@ -8,7 +13,7 @@
 // unit), tcgen05.mma forms S = Q K^T in tensor memory, 128 threads (one per query row) run
 // the online softmax in fp32 straight out of tensor memory, write P back to tensor memory
 // as bf16, and a second tcgen05.mma accumulates O += P V with P read from tensor memory.
-// With rope_theta > 0 the Q and K tiles are rotated in shared memory right after they land.
+// The Q and K tiles are rotated in shared memory right after they land.
 #include <cuda_bf16.h>
 
 #include "pk_common.cuh"

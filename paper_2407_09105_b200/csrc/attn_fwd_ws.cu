@@ -1,7 +1,8 @@
-// Warp-specialised forward kernel (no fused RoPE, query heads per kv head even) for sm_100a.
+// Warp-specialised forward kernel for sm_100a.  Q and K are read as given (no RoPE, or the caller's
+// rotated fp16 copies); any number of query heads per kv head.
 //
 // One CTA per SM works on TWO query tiles at a time: the same block of <= 128 query rows for two
-// adjacent query heads of one kv head.  Both tiles read the same K and V tiles, so each K/V
+// adjacent query heads of one kv head (or two query blocks of one head: see FwdUnit).  Both tiles read the same K and V tiles, so each K/V
 // tile is brought into shared memory once for both, and while the softmax warps of one tile
 // are busy the tensor pipe runs the contractions of the other (ping-pong):
 //   warps 0-3   softmax of tile 0 (one thread per query row, whole row in registers)
