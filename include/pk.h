@@ -19,7 +19,11 @@
  *     the device can see (negative position ids, a pipeline wait that ran out) are
  *     recorded in the workspace's status word; the kernels then stop early and leave
  *     the outputs untouched.  Read it with pk_status_read.
- *   - Supported shapes: D in {64, 128}; Hq % Hkv == 0; 0 <= T; T*Hq*D < 2^31.
+ *   - Supported shapes: D a multiple of 16 up to 128; Hq % Hkv == 0; 0 <= T; T*Hq*D' < 2^31
+ *     with D' = 64 for D <= 64, else 128.  The kernels are built for D = 64 and D = 128; any
+ *     other D runs on zero-padded copies of the tensors kept in the workspace (which
+ *     pk_workspace_bytes sizes for them): one extra streaming pass over every tensor each way
+ *     and contractions at the padded size, same results.
  *   - Query head h reads kv head h / (Hq / Hkv).
  *   - Values of OTHER examples must be finite: a masked probability is exactly 0, but
  *     0 * Inf is NaN inside a tensor-core contraction.
@@ -139,7 +143,9 @@ int pk_rope_apply(void* x, const int32_t* position_ids, int32_t T, int32_t H, in
  *                 rope_theta > 0 the forward leaves rotated copies of q and k in the workspace
  *                 (default RoPE mode); the flag says that they are
  *                 still there (same q, k, position_ids, rope_theta; workspace untouched since
- *                 the forward), so the backward does not make them again.
+ *                 the forward), so the backward does not make them again.  For a padded head
+ *                 size the flag covers the forward's padded copies of q, k and v in the same
+ *                 way (with or without RoPE).
  */
 #define PK_REUSE_PLAN     1
 #define PK_REUSE_ROTATED  2
@@ -187,8 +193,10 @@ int pk_status_read(const void* workspace, void* stream, int32_t* code, int32_t* 
  *       workspace (it reuses the PK_WS_DQ_ACC section), then the warp-specialised kernels run
  *       on them and rotate dQ/dK back in their epilogues.  A K tile is visited by every query
  *       tile of every head of its group, so rotating once costs one HBM pass instead of one
- *       rotation per visit.  Needs D == 128 and an even Hq/Hkv; other shapes use the in-tile mode.
- *   PK_ROPE_IN_TILE  the Q/K tiles are rotated in shared memory right after their TMA load.
+ *       rotation per visit.  Every supported shape.
+ *   PK_ROPE_IN_TILE  the Q/K tiles are rotated in shared memory right after their TMA load
+ *       (D = 64 and 128 only: padded head sizes always take the rotated copies; no sliding
+ *       window).
  */
 #define PK_ROPE_ROTATED_COPIES 0
 #define PK_ROPE_IN_TILE        1

@@ -13,7 +13,8 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libpk.so")
-SOURCES = ["api.cu", "collate.cu", "loss.cu", "plan.cu", "rope.cu", "attn_fwd.cu", "attn_fwd_ws.cu", "attn_bwd.cu", "attn_bwd_ws.cu"]
+SOURCES = ["api.cu", "collate.cu", "loss.cu", "plan.cu", "rope.cu", "attn_fwd.cu", "attn_fwd_ws.cu", "attn_bwd.cu", "attn_bwd_ws.cu",
+           "head_pad.cu"]
 
 
 def _nvcc() -> str:

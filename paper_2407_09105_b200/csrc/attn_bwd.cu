@@ -484,6 +484,24 @@ int launch_bwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& 
 }
 
 }  // namespace
+
+int delta_launch(const void* dout, const void* out, int out_dtype, float* delta, int T, int Hq, int D,
+                 cudaStream_t stream) {
+  const int64_t rows = (int64_t)T * Hq;
+  const int warps = 8;
+  const int64_t rows_per_block = (int64_t)warps * (32 / (D >> 3));
+  const unsigned blocks = (unsigned)((rows + rows_per_block - 1) / rows_per_block);
+  TimedLaunch timed(PK_KERNEL_DELTA, stream);
+  if (out_dtype == PK_BF16)
+    delta_kernel<__nv_bfloat16><<<blocks, warps * 32, 0, stream>>>(
+        static_cast<const __nv_bfloat16*>(dout), static_cast<const __nv_bfloat16*>(out), delta, T,
+        Hq, D);
+  else
+    delta_kernel<float><<<blocks, warps * 32, 0, stream>>>(
+        static_cast<const __nv_bfloat16*>(dout), static_cast<const float*>(out), delta, T, Hq, D);
+  return launch_status();
+}
+
 }  // namespace pk
 
 extern "C" int pk_attn_bwd(const void* dout, const void* q, const void* k, const void* v,
@@ -513,6 +531,10 @@ extern "C" int pk_attn_bwd(const void* dout, const void* q, const void* k, const
   if (!aligned16(dout) || !aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out) ||
       !aligned16(dq) || !aligned16(dk) || !aligned16(dv))
     return PK_ERR_INVALID_ARG;
+  if (D != padded_head_dim(D))
+    return attn_bwd_padded(dout, q, k, v, out, out_dtype, lse, position_ids, T, Hq, Hkv, D,
+                           softmax_scale, rope_theta, window, dq, dk, dv, grad_dtype, reuse_plan,
+                           workspace, workspace_bytes, stream_);
 
   char* ws = static_cast<char*>(workspace);
   int rc;
@@ -532,25 +554,11 @@ extern "C" int pk_attn_bwd(const void* dout, const void* q, const void* k, const
   float* dq_acc = reinterpret_cast<float*>(ws + lay.off[PK_WS_DQ_ACC]);
 
   // (1) delta pre-pass and a cleared dQ accumulator
-  {
-    const int64_t rows = (int64_t)T * Hq;
-    const int warps = 8;
-    const int64_t rows_per_block = (int64_t)warps * (32 / (D >> 3));
-    const unsigned blocks = (unsigned)((rows + rows_per_block - 1) / rows_per_block);
-    TimedLaunch timed(PK_KERNEL_DELTA, stream);
-    if (out_dtype == PK_BF16)
-      delta_kernel<__nv_bfloat16><<<blocks, warps * 32, 0, stream>>>(
-          static_cast<const __nv_bfloat16*>(dout), static_cast<const __nv_bfloat16*>(out), delta,
-          T, Hq, D);
-    else
-      delta_kernel<float><<<blocks, warps * 32, 0, stream>>>(
-          static_cast<const __nv_bfloat16*>(dout), static_cast<const float*>(out), delta, T, Hq, D);
-    if ((rc = launch_status()) != PK_OK) return rc;
-    // only the in-tile RoPE kernel accumulates dQ with reductions and needs a cleared buffer
-    if (use_rope && !rotated_copies &&
-        cudaMemsetAsync(dq_acc, 0, sizeof(float) * (size_t)T * Hq * D, stream) != cudaSuccess)
-      return PK_ERR_CUDA;
-  }
+  if ((rc = delta_launch(dout, out, out_dtype, delta, T, Hq, D, stream)) != PK_OK) return rc;
+  // only the in-tile RoPE kernel accumulates dQ with reductions and needs a cleared buffer
+  if (use_rope && !rotated_copies &&
+      cudaMemsetAsync(dq_acc, 0, sizeof(float) * (size_t)T * Hq * D, stream) != cudaSuccess)
+    return PK_ERR_CUDA;
 
   // (2) main kernel
   CUtensorMap tq, tk, tv, tdo;

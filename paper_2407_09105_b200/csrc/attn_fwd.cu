@@ -360,6 +360,9 @@ extern "C" int pk_attn_fwd(const void* q, const void* k, const void* v,
   if (!q || !k || !v || !position_ids || !out || !lse) return PK_ERR_INVALID_ARG;
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out))
     return PK_ERR_INVALID_ARG;
+  if (D != padded_head_dim(D))
+    return attn_fwd_padded(q, k, v, position_ids, T, Hq, Hkv, D, softmax_scale, rope_theta, window,
+                           out, out_dtype, lse, reuse_plan, workspace, workspace_bytes, stream_);
 
   char* ws = static_cast<char*>(workspace);
   if (!(reuse_plan & PK_REUSE_PLAN)) {

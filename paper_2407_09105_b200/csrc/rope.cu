@@ -36,12 +36,15 @@ __global__ void rope_table_kernel(const int32_t* __restrict__ pos, int T, int D,
 // epilogues of the rotated-copies path read.  Half the bytes of a (cos, sin) pair per entry, which
 // is what their row-per-thread loads are bound by; they take sine and cosine with the fast
 // intrinsics, accurate to 4e-7 on that range.
-__global__ void rope_angle_kernel(const int32_t* __restrict__ pos, int T, int D, double log2_theta,
-                                  float* __restrict__ angle) {
-  const int half = D / 2;
+__global__ void rope_angle_kernel(const int32_t* __restrict__ pos, int T, int D, int row,
+                                  double log2_theta, float* __restrict__ angle) {
   const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (idx >= (int64_t)T * half) return;
-  const int t = (int)(idx / half), i = (int)(idx % half);
+  if (idx >= (int64_t)T * row) return;
+  const int t = (int)(idx / row), i = (int)(idx % row);
+  if (i >= D / 2) {       // columns a padded head does not have
+    angle[idx] = 0.f;
+    return;
+  }
   const double a = (double)pos[t] * exp2(-2.0 * (double)i / (double)D * log2_theta);
   const double two_pi = 6.283185307179586476925286766559;
   angle[idx] = (float)(a - two_pi * rint(a / two_pi));
@@ -137,12 +140,14 @@ int rope_rotate_f16_launch(const void* x, const int32_t* position_ids, int32_t T
 }
 
 int rope_angle_launch(const int32_t* position_ids, int32_t T, int32_t D, float theta,
-                      float* angle, cudaStream_t stream) {
+                      float* angle, cudaStream_t stream, int32_t row) {
   if (T == 0) return PK_OK;
-  const int64_t n = (int64_t)T * (D / 2);
+  if (row <= 0) row = D / 2;
+  const int64_t n = (int64_t)T * row;
   const int threads = 256;
   const unsigned blocks = (unsigned)((n + threads - 1) / threads);
-  rope_angle_kernel<<<blocks, threads, 0, stream>>>(position_ids, T, D, log2((double)theta), angle);
+  rope_angle_kernel<<<blocks, threads, 0, stream>>>(position_ids, T, D, row, log2((double)theta),
+                                                    angle);
   return launch_status();
 }
 

@@ -34,7 +34,10 @@ def test_host_only_calls():
     from paper_2407_09105_b200 import api
     assert api.pk_tile_shape() == (128, 128)
     assert api.pk_workspace_bytes(512, 4, 4, 64) > 0
-    assert api.pk_workspace_bytes(512, 4, 4, 80) == 0          # unsupported head_dim
+    assert api.pk_workspace_bytes(512, 4, 4, 72) == 0          # head_dim not a multiple of 16
+    assert api.pk_workspace_bytes(512, 4, 4, 256) == 0
+    # other head sizes run padded: the padded size's workspace plus room for the copies
+    assert api.pk_workspace_bytes(512, 4, 4, 80) > api.pk_workspace_bytes(512, 4, 4, 128)
     assert api.pk_workspace_bytes(512, 6, 4, 64) == 0          # Hq % Hkv != 0
     assert api.pk_workspace_bytes(-1, 4, 4, 64) == 0
     offs = [api.pk_workspace_section(s, 1000, 8, 2, 128) for s in range(8)]
@@ -50,7 +53,7 @@ def test_argument_validation_returns_codes_without_a_gpu():
     L = api.lib()
     # null workspace / negative T / unsupported shapes are rejected before any CUDA call
     assert L.pk_seqlens_from_posids(None, -1, None, None, None, None, 0, None) == api.PK_ERR_INVALID_ARG
-    assert L.pk_attn_fwd(None, None, None, None, 16, 4, 4, 80, 1.0, 0.0, 0, None, 0, None, 0, None, 0,
+    assert L.pk_attn_fwd(None, None, None, None, 16, 4, 4, 72, 1.0, 0.0, 0, None, 0, None, 0, None, 0,
                          None) == api.PK_ERR_UNSUPPORTED
     assert L.pk_attn_fwd(None, None, None, None, 16, 4, 4, 64, -1.0, 0.0, 0, None, 0, None, 0, None, 0,
                          None) == api.PK_ERR_INVALID_ARG
