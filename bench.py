@@ -37,7 +37,11 @@ UNIT = "TFLOP/s"
 
 # DRAM bytes per causal (query, key, q-head) pair of the dominant (dK/dV) kernel, from the ncu
 # capture summarised in profiles/ (scaled to a launch by the number of pairs); None = not captured.
-NCU_BWD_DRAM_BYTES_PER_PAIR = 0.3330   # attn_bwd_dkv_kernel, profiles/attn_kernels_c4_2packs.txt
+# DRAM bytes per (causal pair, q head) of one launch on the full c4 workload
+# (profiles/attn_kernels_c4_full_dram_bytes.txt); other workloads are scaled by their pair count
+NCU_BWD_DRAM_BYTES_PER_PAIR = 0.3838   # attn_bwd_dkv_kernel
+NCU_DQ_DRAM_BYTES_PER_PAIR = 0.3408    # attn_bwd_dq_kernel
+NCU_FWD_DRAM_BYTES_PER_PAIR = 0.2432   # attn_fwd_ws_kernel
 
 
 def _peaks():
@@ -568,28 +572,41 @@ def main():
     peaks = _peaks()
     if calls_per_step > 1:      # per-kernel events are recorded for the flat run only
         fwd_ms = bwd_ms = dq_ms = float('nan')
-    # without fused RoPE the backward is two kernels: dK/dV (6 of the 10 useful FLOPs per pair and
-    # head-dim: dV, dK, plus one of the two recomputed products) and dQ.  The dominant kernel is
-    # the dK/dV one; its useful work is dV and dK only: 4*D FLOPs per pair.
-    bwd_flops = (w.useful_flops_bwd * 4 // 10) if split else w.useful_flops_bwd
-    bwd_tflops = bwd_flops / (bwd_ms * 1e-3) / 1e12
-    executed = ((8 if split else 10) * D * Hq * w.causal_pairs) / (bwd_ms * 1e-3) / 1e12
+    # The backward (10*D FLOPs per causal pair and q head: S, dP, dV, dK, dQ) dominates the step.
+    # Without in-tile RoPE it runs as two launches, dK/dV (S, dP, dV, dK: 8*D) and dQ (S and dP once
+    # more, and dQ: 6*D executed, 2*D of them new), so the roofline entry takes the two together:
+    # the paper's 10*D per pair over the sum of their durations.  The per-launch figures follow.
+    bwd_both_ms = bwd_ms + dq_ms
+    bwd_tflops = w.useful_flops_bwd / (bwd_both_ms * 1e-3) / 1e12
+    per_pair = Hq * w.causal_pairs
     fwd_tflops = w.useful_flops_fwd / (fwd_ms * 1e-3) / 1e12
+    traffic = None
+    if split and NCU_BWD_DRAM_BYTES_PER_PAIR is not None and NCU_DQ_DRAM_BYTES_PER_PAIR is not None:
+        traffic = (NCU_BWD_DRAM_BYTES_PER_PAIR + NCU_DQ_DRAM_BYTES_PER_PAIR) * per_pair
     roofline = {
-        "kernel": "attn_bwd_dkv_kernel" if split else "attn_bwd_kernel", "bound": "tensor", "achieved": bwd_tflops,
+        "kernel": ("attn_bwd_dkv_kernel + attn_bwd_dq_kernel (the backward)" if split
+                   else "attn_bwd_kernel"),
+        "bound": "tensor", "achieved": bwd_tflops,
         "peak": peaks["sustained"], "peak_kind": f"bf16 sustained, {peaks['source']}",
         "peak_burst": peaks["burst"], "unit": "TFLOP/s", "frac": bwd_tflops / peaks["sustained"],
-        "traffic": (None if (NCU_BWD_DRAM_BYTES_PER_PAIR is None or not split)
-                    else NCU_BWD_DRAM_BYTES_PER_PAIR * w.causal_pairs * Hq),
-        "ms_per_launch": bwd_ms,
-        "note": ("dK/dV kernel: useful = dV and dK (4*D FLOPs per causal pair and head); it also "
-                 "recomputes S and dP, executed_tflops counts those" if split else "fused-RoPE kernel"),
-        "executed_tflops": executed,
-        "bwd_dq_kernel": ({"achieved": (w.useful_flops_bwd * 2 // 10) / (dq_ms * 1e-3) / 1e12,
-                           "executed_tflops": (6 * D * Hq * w.causal_pairs) / (dq_ms * 1e-3) / 1e12,
-                           "ms_per_launch": dq_ms} if split else None),
+        "traffic": traffic, "ms_per_launch": bwd_both_ms, "launches_per_step": 2 if split else 1,
+        "note": ("algorithmic FLOPs = 10*D per causal pair and q head over both launches; each "
+                 "launch's own figures below count what it executes" if split else "in-tile RoPE kernel"),
+        "bwd_dkv_kernel": ({"executed_tflops": 8 * D * per_pair / (bwd_ms * 1e-3) / 1e12,
+                            "frac_executed": 8 * D * per_pair / (bwd_ms * 1e-3) / 1e12 / peaks["sustained"],
+                            "ms_per_launch": bwd_ms,
+                            "traffic": (None if NCU_BWD_DRAM_BYTES_PER_PAIR is None
+                                        else NCU_BWD_DRAM_BYTES_PER_PAIR * per_pair)}
+                           if split else None),
+        "bwd_dq_kernel": ({"executed_tflops": 6 * D * per_pair / (dq_ms * 1e-3) / 1e12,
+                           "frac_executed": 6 * D * per_pair / (dq_ms * 1e-3) / 1e12 / peaks["sustained"],
+                           "ms_per_launch": dq_ms,
+                           "traffic": (None if NCU_DQ_DRAM_BYTES_PER_PAIR is None
+                                       else NCU_DQ_DRAM_BYTES_PER_PAIR * per_pair)}
+                          if split else None),
         "fwd_kernel": {"achieved": fwd_tflops, "frac": fwd_tflops / peaks["sustained"],
-                       "ms_per_launch": fwd_ms},
+                       "ms_per_launch": fwd_ms,
+                       "traffic": NCU_FWD_DRAM_BYTES_PER_PAIR * per_pair if split else None},
     }
     cpu_baseline = None
     if not args.no_cpu_baseline:
