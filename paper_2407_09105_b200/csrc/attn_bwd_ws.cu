@@ -521,8 +521,14 @@ enum DqBar {
 // They are copied once per unit from shared memory into tensor memory, so that those two
 // contractions read only K / V from shared memory (the shared-memory port, not the tensor
 // pipe, was the bound when all four operands came from there).
+// Warps: 0-7 compute, 8 issues the contractions, 9 loads, 10-11 idle, 12-15 write each unit's dQ
+// (one thread per query row) while the compute warps are already in the next unit.  Registers
+// are handed from the small roles to the compute warps at the start (setmaxnreg).
+constexpr int kDqThreads = 512;
+constexpr int kDqEpiWarp0 = 12;
+constexpr int kDqEpiThreads = 128;
 template <int D, bool kRot, typename GradT>
-__global__ void __launch_bounds__(kWsThreads, 1)
+__global__ void __launch_bounds__(kDqThreads, 1)
 attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                    const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_do,
                    const int4* __restrict__ items, const int32_t* __restrict__ order, int32_t* hdr,
@@ -550,7 +556,7 @@ attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
     mbar_init(bar(dqDpFull), 1);
     mbar_init(bar(dqDsReady), kComputeThreads);
     mbar_init(bar(dqDone), 1);
-    mbar_init(bar(dqRead), kComputeThreads);
+    mbar_init(bar(dqRead), kDqEpiThreads);
     for (int i = 0; i < kUnitRing; ++i) mbar_init(bar(dqUnitFull0 + i), 1);
     fence_mbar_init();
     *s_abort = ((sbase & 1023u) != 0) ? 1 : 0;
@@ -578,6 +584,10 @@ attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
     return (window > 0 && reach > 0) ? reach / kBN : 0;
   };
 
+  // Register budget: 512 threads start with 128 each; the compute warps need more, the rest less.
+  // Each warpgroup changes its allowance at the top of its own branch.
+  if ((warp >> 2) == (kMmaWarp >> 2)) {
+  setmaxnreg_dec<40>();
   if (warp == kLoadWarp) {
     // =============================== loader ===============================================
     if (lane == 0) {
@@ -702,8 +712,10 @@ attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         __syncwarp();
       }
     }
-  } else {
+  }
+  } else if (warp < kMmaWarp) {
     // =============================== compute ===============================================
+    setmaxnreg_inc<176>();
     const int row = tid & 127;              // query row inside the tile
     const int qd = tid >> 7;                // which group of kCW key columns
     const uint32_t lane_off = static_cast<uint32_t>((warp & 3) * 32) << 16;
@@ -804,57 +816,76 @@ attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
       // The last S and dP of this unit have been consumed, so Q/dO of the NEXT unit can move into
       // tensor memory now; the issuing warp then starts that unit while this one's dQ is written.
       if (unit_at(uc + 1) < n_units && !*s_abort) copy_q_do(uc + 1);
-      // ---- unit epilogue: dQ rows, scaled (column groups 0 and 1 write half a row each) -----
+    }
+  } else if (warp >= kDqEpiWarp0) {
+    // =============================== dQ writer =============================================
+    // One thread per query row: waits for the unit's last contraction, pulls the row of dQ out of
+    // tensor memory 32 columns at a time, scales (and rotates back), stores.  The accumulator is
+    // released as soon as the last columns are in registers.
+    setmaxnreg_dec<96>();
+    const int row = tid & 127;
+    const uint32_t lane_off = static_cast<uint32_t>((warp & 3) * 32) << 16;
+    for (int uc = 0;; ++uc) {
+      mbar_wait(bar(dqUnitFull0 + uc % kUnitRing), (uc / kUnitRing) & 1, s_abort);
+      const int u = static_cast<int>(s_unit[uc % kUnitRing]);
+      if (u >= n_units || *s_abort) break;
+      const int4 it = items[order[u / Hq]];
+      const int h = u % Hq;
+      const int tok = it.x + row;
       mbar_wait(bar(dqDone), uc & 1, s_abort);
       tc_fence_after();
-      if (qd < 2) {
-        const bool live = (row < q_len) && (*s_abort == 0);
-        if (kRot) {
-          // rotate back by -angle: this thread owns pairs i in [32*qd, +32) and i + D/2 (with
-          // D = 64 there are only 32 pairs: column group 0 takes them all)
-          static_assert(!kRot || D == 128 || D == 64, "rotated path is built for D = 64 and 128");
-          GradT* dst = dq + ((size_t)tok * Hq + h) * D + qd * 32;
+      const bool live = (row < it.y) && (*s_abort == 0);
+      GradT* dst = dq + ((size_t)tok * Hq + h) * D;
+      if (kRot) {
+        // rotate back by -angle: pairs (i, i + D/2), 32 of them at a time
+        static_assert(!kRot || D == 128 || D == 64, "rotated path is built for D = 64 and 128");
+        const float* cs = rope_angle + (size_t)tok * (D / 2);
+#pragma unroll
+        for (int c = 0; c < D / 2; c += 32) {
           uint32_t x1[32], x2[32];
-          float y1[32], y2[32];
-          const bool mine = qd * 32 < D / 2;
-          if (mine) {
-            tmem_ld32(tdQ + lane_off + qd * 32, x1);
-            tmem_ld32(tdQ + lane_off + D / 2 + qd * 32, x2);
-          }
+          tmem_ld32(tdQ + lane_off + c, x1);
+          tmem_ld32(tdQ + lane_off + D / 2 + c, x2);
           tmem_wait_ld();
-          if (live && mine) {
-            const float* cs = rope_angle + (size_t)tok * (D / 2) + qd * 32;
+          if (c + 32 >= D / 2) {
+            tc_fence_before();
+            mbar_arrive(bar(dqRead));
+          }
+          if (live) {
+            float y1[32], y2[32];
 #pragma unroll
             for (int e4 = 0; e4 < 32; e4 += 8) {
               float2 t4[8];
-              ld_angles8(cs + e4, t4);
+              ld_angles8(cs + c + e4, t4);
 #pragma unroll
               for (int k = 0; k < 8; ++k) {
                 const int e = e4 + k;
-                const float a = __uint_as_float(x1[e]) * scale, b = __uint_as_float(x2[e]) * scale;
-                y1[e] = a * t4[k].x + b * t4[k].y;
-                y2[e] = b * t4[k].x - a * t4[k].y;
+                const float a = __uint_as_float(x1[e]) * scale, bb = __uint_as_float(x2[e]) * scale;
+                y1[e] = a * t4[k].x + bb * t4[k].y;
+                y2[e] = bb * t4[k].x - a * t4[k].y;
               }
             }
-            store_chunk32<GradT>(dst, y1);
-            store_chunk32<GradT>(dst + D / 2, y2);
+            store_chunk32<GradT>(dst + c, y1);
+            store_chunk32<GradT>(dst + D / 2 + c, y2);
           }
-        } else {
-          GradT* dst = dq + ((size_t)tok * Hq + h) * D + qd * (D / 2);
+        }
+      } else {
 #pragma unroll
-          for (int c = 0; c < D / 64; ++c) {
-            uint32_t x[32];
+        for (int c = 0; c < D; c += 32) {
+          uint32_t x[32];
+          tmem_ld32(tdQ + lane_off + c, x);
+          tmem_wait_ld();
+          if (c + 32 >= D) {
+            tc_fence_before();
+            mbar_arrive(bar(dqRead));
+          }
+          if (live) {
             float y[32];
-            tmem_ld32(tdQ + lane_off + qd * (D / 2) + c * 32, x);
-            tmem_wait_ld();
 #pragma unroll
             for (int e = 0; e < 32; ++e) y[e] = __uint_as_float(x[e]) * scale;
-            if (live) store_chunk32<GradT>(dst + c * 32, y);
+            store_chunk32<GradT>(dst + c, y);
           }
         }
       }
-      tc_fence_before();
-      mbar_arrive(bar(dqRead));
     }
   }
 
@@ -895,7 +926,7 @@ int launch_ws(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& t
   if (launch_status() != PK_OK) return PK_ERR_CUDA;
   {
     TimedLaunch timed(PK_KERNEL_BWD_DQ, stream);
-    kern_q<<<grid, kWsThreads, DqSmem<D>::kTotal, stream>>>(
+    kern_q<<<grid, kDqThreads, DqSmem<D>::kTotal, stream>>>(
         tq, tk, tv, tdo, reinterpret_cast<const int4*>(ws + lay.off[PK_WS_FWD_ITEMS]),
         reinterpret_cast<const int32_t*>(ws + lay.off[PK_WS_FWD_ORDER]), hdr, lse, delta,
         static_cast<GradT*>(dq), table, T, Hq, Hkv, scale, scale * kLog2eWs, window);

@@ -95,6 +95,18 @@ __device__ __forceinline__ void tmem_alloc(uint32_t smem_result, uint32_t ncols)
   asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
                ::"r"(smem_result), "r"(ncols) : "memory");
 }
+// Register reallocation between the warpgroups of a CTA: every warp of a warpgroup (4 consecutive
+// warps) executes the same one.  inc waits until the registers are there, so the decs of the
+// other warpgroups must not depend on anything.
+template <int N>
+__device__ __forceinline__ void setmaxnreg_inc() {
+  asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N));
+}
+template <int N>
+__device__ __forceinline__ void setmaxnreg_dec() {
+  asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N));
+}
+
 __device__ __forceinline__ void tmem_relinquish() {
   asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
 }
