@@ -56,11 +56,8 @@ __device__ __forceinline__ void store_chunk32<float>(float* dst, const float* x)
   for (int c = 0; c < 32; c += 4)
     *reinterpret_cast<float4*>(dst + c) = make_float4(x[c], x[c + 1], x[c + 2], x[c + 3]);
 }
-template <>
-__device__ __forceinline__ void store_chunk32<__nv_bfloat16>(__nv_bfloat16* dst, const float* x) {
-  uint32_t v[16];
-#pragma unroll
-  for (int c = 0; c < 16; ++c) v[c] = pack_bf16x2(x[2 * c], x[2 * c + 1]);
+// 32 bf16 values, already packed in pairs
+__device__ __forceinline__ void store_packed32(__nv_bfloat16* dst, const uint32_t* v) {
   if ((reinterpret_cast<uintptr_t>(dst) & 31) == 0) {
     st_global_v8(dst, v);
     st_global_v8(dst + 16, v + 8);
@@ -69,6 +66,13 @@ __device__ __forceinline__ void store_chunk32<__nv_bfloat16>(__nv_bfloat16* dst,
 #pragma unroll
   for (int c = 0; c < 16; c += 4)
     *reinterpret_cast<uint4*>(dst + 2 * c) = make_uint4(v[c], v[c + 1], v[c + 2], v[c + 3]);
+}
+template <>
+__device__ __forceinline__ void store_chunk32<__nv_bfloat16>(__nv_bfloat16* dst, const float* x) {
+  uint32_t v[16];
+#pragma unroll
+  for (int c = 0; c < 16; ++c) v[c] = pack_bf16x2(x[2 * c], x[2 * c + 1]);
+  store_packed32(dst, v);
 }
 
 

@@ -9,6 +9,9 @@
 //   warps 4-7   softmax of tile 1
 //   warp  8     issues every tcgen05.mma:  S_t = Q_t K^T  and  O_t += P_t V  (P_t from tensor memory)
 //   warp  9     TMA: the two Q tiles per unit, K/V tiles through a 2-stage ring
+//   warps 12-15 write O_0 and then O_1 of each unit (one thread per row) while the softmax warps
+//               are already in the next unit; warps 10-11 idle.  Registers move from the small
+//               roles to the softmax warps at the start (setmaxnreg).
 // Tensor memory: [0,128) S_0 / P_0, [128,256) S_1 / P_1, [256,384) O_0, [384,512) O_1.
 // The commit that announces S_t(j) also covers O_t += P_t V of step j-1 (same pipe, in order), so
 // the softmax warps may rescale O_t in tensor memory as soon as they see S_t(j).
@@ -27,7 +30,8 @@ namespace {
 
 using namespace ptx;
 
-constexpr int kFwsThreads = 320;
+constexpr int kFwsThreads = 512;
+constexpr int kFwsEpiWarp0 = 12;
 constexpr int kFwsMmaWarp = 8;
 constexpr int kFwsLoadWarp = 9;
 constexpr float kLog2eF = 1.4426950408889634f;
@@ -51,12 +55,14 @@ struct FwsSmem {
   static constexpr int kStageBytes = 2 * kTileBytes;
   static constexpr int kBars = kKV0 + 2 * kStageBytes;
   static constexpr int kMisc = kBars + 24 * 8;               // tmem base, abort flag, unit ring
-  static constexpr int kTotal = kMisc + 16 + 4 * kFwsUnitRing;
+  static constexpr int kInvL = kMisc + 16 + 4 * kFwsUnitRing;   // [2][128] floats: 1 / row sum
+  static constexpr int kTotal = kInvL + 1024;
 };
 
 enum FwsBar {
   fQFull = 0, fQEmpty, fKvFull0, fKvFull1, fKvEmpty0, fKvEmpty1, fSFull0, fSFull1, fPReady0,
   fPReady1, fOFull0, fOFull1, fORead0, fORead1, fUnitFull0, fUnitFull1, fUnitFull2, fUnitFull3,
+  fLReady0, fLReady1,
   fNumBars
 };
 
@@ -154,6 +160,8 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
     mbar_init(bar(fOFull1), 1);
     mbar_init(bar(fORead0), 128);
     mbar_init(bar(fORead1), 128);
+    mbar_init(bar(fLReady0), 128);
+    mbar_init(bar(fLReady1), 128);
     for (int i = 0; i < kFwsUnitRing; ++i) mbar_init(bar(fUnitFull0 + i), 1);
     fence_mbar_init();
     *s_abort = ((sbase & 1023u) != 0) ? 1 : 0;
@@ -173,6 +181,11 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
   if (!plan_ok && blockIdx.x == 0 && tid == 0) set_status(hdr, PK_ERR_NO_PLAN, T);
   const int n_units = plan_ok ? hdr[PK_HDR_N_ITEMS] * (pair_blocks ? Hq : Hq / 2) : 0;
 
+  float* s_invl = reinterpret_cast<float*>(smem + L::kInvL);
+  // Register budget: 512 threads start with 128 each; every warpgroup changes its allowance at the
+  // top of its own branch.
+  if ((warp >> 2) == (kFwsMmaWarp >> 2)) {
+  setmaxnreg_dec<40>();
   if (warp == kFwsLoadWarp) {
     // =============================== loader ===============================================
     if (lane == 0) {
@@ -282,8 +295,10 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         __syncwarp();
       }
     }
-  } else {
+  }
+  } else if (warp < kFwsMmaWarp) {
     // =============================== softmax (warps 0-3: tile 0, warps 4-7: tile 1) =======
+    setmaxnreg_inc<184>();
     const int t = tid >> 7;
     const int row = tid & 127;
     const uint32_t lane_off = static_cast<uint32_t>((warp & 3) * 32) << 16;
@@ -363,24 +378,46 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         tc_fence_before();
         mbar_arrive(bar(fPReady0 + t));
       }
-      // ---- epilogue: O / l and lse ---------------------------------------------------------
-      mbar_wait(bar(fOFull0 + t), uc & 1, s_abort);
-      tc_fence_after();
-      {
-        const bool live = (row < q_len) && (*s_abort == 0);
-        const float inv_l = 1.f / l_run;
-        if (live) lse[(size_t)h * T + q_start + row] = (m_run + log2f(l_run)) * kLn2F;
-        OutT* orow = out + ((size_t)(q_start + row) * Hq + h) * D;
+      // ---- lse from here; O_t / l is written by the writer warps, which get 1 / l ------------
+      if ((row < q_len) && (*s_abort == 0))
+        lse[(size_t)h * T + q_start + row] = (m_run + log2f(l_run)) * kLn2F;
+      s_invl[t * 128 + row] = 1.f / l_run;
+      mbar_arrive(bar(fLReady0 + t));
+    }
+  } else if (warp >= kFwsEpiWarp0) {
+    // =============================== O writer ==============================================
+    // One thread per query row, tile 0 then tile 1 of every unit: waits for the tile's last
+    // contraction, pulls the row out of tensor memory 32 columns at a time, scales by 1 / l,
+    // stores.  The accumulator is released as soon as its last columns are in registers.
+    setmaxnreg_dec<96>();
+    const int row = tid & 127;
+    const uint32_t lane_off = static_cast<uint32_t>((warp & 3) * 32) << 16;
+    for (int uc = 0;; ++uc) {
+      mbar_wait(bar(fUnitFull0 + uc % kFwsUnitRing), (uc / kFwsUnitRing) & 1, s_abort);
+      const int u = s_unit[uc % kFwsUnitRing];
+      if (u >= n_units || *s_abort) break;
+      const FwdUnit w = decode_fwd_unit(u, items, order, Hq, G, pair_blocks, window);
+#pragma unroll
+      for (int t = 0; t < 2; ++t) {
+        mbar_wait(bar(fLReady0 + t), uc & 1, s_abort);
+        const float inv_l = s_invl[t * 128 + row];
+        mbar_wait(bar(fOFull0 + t), uc & 1, s_abort);
+        tc_fence_after();
+        const bool live = (row < w.q_len[t]) && (*s_abort == 0);
+        const uint32_t tO = tmem + 256 + t * 128 + lane_off;
+        OutT* orow = out + ((size_t)(w.q_start[t] + row) * Hq + w.h[t]) * D;
 #pragma unroll
         for (int c = 0; c < D / 32; ++c) {
           uint32_t o[32];
           tmem_ld32(tO + c * 32, o);
           tmem_wait_ld();
+          if (c == D / 32 - 1) {
+            tc_fence_before();
+            mbar_arrive(bar(fORead0 + t));
+          }
           if (live) store_out32<OutT>(orow + c * 32, o, inv_l);
         }
       }
-      tc_fence_before();
-      mbar_arrive(bar(fORead0 + t));
     }
   }
 
