@@ -42,6 +42,12 @@ constexpr int kComputeThreads = PK_BWD_COMPUTE_THREADS;
 constexpr int kNQ = kComputeThreads / 128;                // column groups per tile row
 constexpr int kCW = 128 / kNQ;                            // columns per compute thread
 constexpr int kWsThreads = kComputeThreads + 64;
+// with the writer warpgroup: warps 0-7 compute, 8 issues the contractions, 9 loads, 10-11 idle,
+// 12-15 write the unit's results while the compute warps are already in the next unit; registers
+// move from the small roles to the compute warps at the start (setmaxnreg)
+constexpr int kBwdThreads = 512;
+constexpr int kWriterWarp0 = 12;
+constexpr int kWriterThreads = 128;
 constexpr int kMmaWarp = kComputeThreads / 32;
 constexpr int kLoadWarp = kMmaWarp + 1;
 static_assert(kNQ == 2, "the dK/dV kernel gives each compute thread 64 query columns");
@@ -93,7 +99,7 @@ static_assert(kvNumBars <= 24, "barrier area");
 // region, and S^T of step n+1 is written there as soon as every thread holds dP^T(n) in
 // registers: the next step's scores never wait for the tensor pipe to consume P^T or dS^T.
 template <int D, bool kRot, typename GradT>
-__global__ void __launch_bounds__(kWsThreads, 1)
+__global__ void __launch_bounds__(kBwdThreads, 1)
 attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                     const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_do,
                     const int4* __restrict__ items, const int32_t* __restrict__ order, int32_t* hdr,
@@ -129,7 +135,7 @@ attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     mbar_init(bar(kvDsReady), kComputeThreads);
     mbar_init(bar(kvDpRead), kComputeThreads);
     mbar_init(bar(kvUnitDone), 1);
-    mbar_init(bar(kvDkvRead), kComputeThreads);
+    mbar_init(bar(kvDkvRead), kWriterThreads);
     for (int i = 0; i < kUnitRing; ++i) mbar_init(bar(kvUnitFull0 + i), 1);
     fence_mbar_init();
     *s_abort = ((sbase & 1023u) != 0) ? 1 : 0;   // swizzled tiles need a 1024-byte aligned base
@@ -157,6 +163,10 @@ attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     return window > 0 ? min(n, (kv_len - 1 + window - 1) / kBM + 1) : n;
   };
 
+  // Register budget: 512 threads start with 128 each; every warpgroup changes its allowance at the
+  // top of its own branch.
+  if ((warp >> 2) == (kMmaWarp >> 2)) {
+  setmaxnreg_dec<40>();
   if (warp == kLoadWarp) {
     // =============================== loader ===============================================
     // Steps are numbered globally (gs) across this CTA's units.  Q(gs) goes to Q stage gs % 3 once
@@ -336,8 +346,10 @@ attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         __syncwarp();
       }
     }
-  } else {
+  }
+  } else if (warp < kMmaWarp) {
     // =============================== compute ===============================================
+    setmaxnreg_inc<176>();
     const int row = tid & 127;              // key row inside the block
     const int qd = tid >> 7;                // this thread's query columns: [64*qd, +64)
     const uint32_t lane_off = static_cast<uint32_t>((warp & 3) * 32) << 16;
@@ -425,62 +437,88 @@ attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           mbar_arrive(bar(kvDsReady));
         }
       }
-      // ---- unit epilogue: the first half of the column groups writes dV, the second dK ------
+    }
+  } else if (warp >= kWriterWarp0) {
+    // =============================== dK / dV writer ========================================
+    // One thread per key row: waits for the unit's last contraction, pulls the rows of dV and dK
+    // out of tensor memory 32 columns at a time, scales dK (and rotates it back), stores.  The
+    // accumulators are released as soon as the last columns are in registers.
+    setmaxnreg_dec<96>();
+    const int row = tid & 127;
+    const uint32_t lane_off = static_cast<uint32_t>((warp & 3) * 32) << 16;
+    for (int uc = 0;; ++uc) {
+      mbar_wait(bar(kvUnitFull0 + uc % kUnitRing), (uc / kUnitRing) & 1, s_abort);
+      const int u = s_unit[uc % kUnitRing];
+      if (u >= n_units || *s_abort) break;
+      const int4 it = items[order[u / Hkv]];
+      const int g = u % Hkv;
+      const int tok = it.x + row;
       mbar_wait(bar(kvUnitDone), uc & 1, s_abort);
       tc_fence_after();
-      {
-        constexpr int kHalfGroups = kNQ / 2;               // groups per output tensor
-        constexpr int kEpiCols = D / kHalfGroups;          // columns each thread writes
-        const bool is_dv = qd < kHalfGroups;
-        const int col0 = (qd % kHalfGroups) * kEpiCols;
-        const bool live = (row < kv_len) && (*s_abort == 0);
-        const int tok = kv_start + row;
-        GradT* dst = (is_dv ? dv : dk) + ((size_t)tok * Hkv + g) * D + col0;
-        const uint32_t src = (is_dv ? tdV : tdK) + lane_off + col0;
-        const float mul = is_dv ? 1.f : scale;
-        if (kRot && !is_dv) {
-          // dK was formed against the rotated k: rotate back by -angle, pairs (i, i + D/2)
-          static_assert(!kRot || kEpiCols == D, "one thread holds both halves of a dK row");
+      const bool live = (row < it.y) && (*s_abort == 0);
+      GradT* dv_row = dv + ((size_t)tok * Hkv + g) * D;
+      GradT* dk_row = dk + ((size_t)tok * Hkv + g) * D;
 #pragma unroll
-          for (int c = 0; c < D / 64; ++c) {
-            uint32_t x1[32], x2[32];
-            float y1[32], y2[32];
-            tmem_ld32(src + c * 32, x1);
-            tmem_ld32(src + D / 2 + c * 32, x2);
-            tmem_wait_ld();
-            if (live) {
-              const float* cs = rope_angle + (size_t)tok * (D / 2) + c * 32;
+      for (int c = 0; c < D; c += 32) {
+        uint32_t x[32];
+        tmem_ld32(tdV + lane_off + c, x);
+        tmem_wait_ld();
+        if (live) {
+          float y[32];
 #pragma unroll
-              for (int e4 = 0; e4 < 32; e4 += 8) {
-                float2 t4[8];
-                ld_angles8(cs + e4, t4);
+          for (int e = 0; e < 32; ++e) y[e] = __uint_as_float(x[e]);
+          store_chunk32<GradT>(dv_row + c, y);
+        }
+      }
+      if (kRot) {
+        // dK was formed against the rotated k: rotate back by -angle, pairs (i, i + D/2)
+        const float* cs = rope_angle + (size_t)tok * (D / 2);
 #pragma unroll
-                for (int k = 0; k < 8; ++k) {
-                  const int e = e4 + k;
-                  const float a = __uint_as_float(x1[e]) * mul, b = __uint_as_float(x2[e]) * mul;
-                  y1[e] = a * t4[k].x + b * t4[k].y;
-                  y2[e] = b * t4[k].x - a * t4[k].y;
-                }
-              }
-              store_chunk32<GradT>(dst + c * 32, y1);
-              store_chunk32<GradT>(dst + D / 2 + c * 32, y2);
-            }
+        for (int c = 0; c < D / 2; c += 32) {
+          uint32_t x1[32], x2[32];
+          tmem_ld32(tdK + lane_off + c, x1);
+          tmem_ld32(tdK + lane_off + D / 2 + c, x2);
+          tmem_wait_ld();
+          if (c + 32 >= D / 2) {
+            tc_fence_before();
+            mbar_arrive(bar(kvDkvRead));
           }
-        } else {
+          if (live) {
+            float y1[32], y2[32];
 #pragma unroll
-          for (int c = 0; c < kEpiCols / 32; ++c) {
-            uint32_t x[32];
+            for (int e4 = 0; e4 < 32; e4 += 8) {
+              float2 t4[8];
+              ld_angles8(cs + c + e4, t4);
+#pragma unroll
+              for (int k = 0; k < 8; ++k) {
+                const int e = e4 + k;
+                const float p = __uint_as_float(x1[e]) * scale, q = __uint_as_float(x2[e]) * scale;
+                y1[e] = p * t4[k].x + q * t4[k].y;
+                y2[e] = q * t4[k].x - p * t4[k].y;
+              }
+            }
+            store_chunk32<GradT>(dk_row + c, y1);
+            store_chunk32<GradT>(dk_row + D / 2 + c, y2);
+          }
+        }
+      } else {
+#pragma unroll
+        for (int c = 0; c < D; c += 32) {
+          uint32_t x[32];
+          tmem_ld32(tdK + lane_off + c, x);
+          tmem_wait_ld();
+          if (c + 32 >= D) {
+            tc_fence_before();
+            mbar_arrive(bar(kvDkvRead));
+          }
+          if (live) {
             float y[32];
-            tmem_ld32(src + c * 32, x);
-            tmem_wait_ld();
 #pragma unroll
-            for (int e = 0; e < 32; ++e) y[e] = __uint_as_float(x[e]) * mul;
-            if (live) store_chunk32<GradT>(dst + c * 32, y);
+            for (int e = 0; e < 32; ++e) y[e] = __uint_as_float(x[e]) * scale;
+            store_chunk32<GradT>(dk_row + c, y);
           }
         }
       }
-      tc_fence_before();
-      mbar_arrive(bar(kvDkvRead));
     }
   }
 
@@ -521,12 +559,10 @@ enum DqBar {
 // They are copied once per unit from shared memory into tensor memory, so that those two
 // contractions read only K / V from shared memory (the shared-memory port, not the tensor
 // pipe, was the bound when all four operands came from there).
-// Warps: 0-7 compute, 8 issues the contractions, 9 loads, 10-11 idle, 12-15 write each unit's dQ
-// (one thread per query row) while the compute warps are already in the next unit.  Registers
-// are handed from the small roles to the compute warps at the start (setmaxnreg).
-constexpr int kDqThreads = 512;
-constexpr int kDqEpiWarp0 = 12;
-constexpr int kDqEpiThreads = 128;
+// Warps as in the dK/dV kernel: 12-15 write each unit's dQ (one thread per query row).
+constexpr int kDqThreads = kBwdThreads;
+constexpr int kDqEpiWarp0 = kWriterWarp0;
+constexpr int kDqEpiThreads = kWriterThreads;
 template <int D, bool kRot, typename GradT>
 __global__ void __launch_bounds__(kDqThreads, 1)
 attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
@@ -917,7 +953,7 @@ int launch_ws(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& t
     return PK_ERR_CUDA;
   {
     TimedLaunch timed(PK_KERNEL_BWD, stream);
-    kern_kv<<<grid, kWsThreads, DkvSmem<D>::kTotal, stream>>>(
+    kern_kv<<<grid, kBwdThreads, DkvSmem<D>::kTotal, stream>>>(
         tq, tk, tv, tdo, reinterpret_cast<const int4*>(ws + lay.off[PK_WS_BWD_ITEMS]),
         reinterpret_cast<const int32_t*>(ws + lay.off[PK_WS_BWD_ORDER]), hdr, lse, delta,
         static_cast<GradT*>(dk), static_cast<GradT*>(dv), table, T, Hq, Hkv, scale,
