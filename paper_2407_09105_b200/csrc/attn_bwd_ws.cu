@@ -20,7 +20,10 @@
 // Roles: 8 compute warps (lane = tensor-memory row; warp w works on columns [64*(w/4), +64) of
 // the rows of lane quarter w%4; 16 warps of 32 columns measured slightly slower because they
 // take issue slots from the warp that feeds the tensor pipe), one warp that walks the MMA
-// schedule with one elected lane issuing every tcgen05.mma, one warp that drives TMA.
+// schedule with one elected lane issuing every tcgen05.mma, one warp that drives TMA, and four
+// writer warps (one thread per row) that scale, rotate back and store a unit's accumulators
+// while the compute warps are already in the next unit.  512 threads start with 128 registers
+// each; setmaxnreg moves them to the compute warps at the top of each warpgroup's branch.
 // Units are drawn from a counter (see kUnitRing below) in the plan's order.
 // Every wait is bounded; on expiry an abort flag makes all later waits return at once.
 #include <cuda_bf16.h>
@@ -41,10 +44,7 @@ using namespace ptx;
 constexpr int kComputeThreads = PK_BWD_COMPUTE_THREADS;
 constexpr int kNQ = kComputeThreads / 128;                // column groups per tile row
 constexpr int kCW = 128 / kNQ;                            // columns per compute thread
-constexpr int kWsThreads = kComputeThreads + 64;
-// with the writer warpgroup: warps 0-7 compute, 8 issues the contractions, 9 loads, 10-11 idle,
-// 12-15 write the unit's results while the compute warps are already in the next unit; registers
-// move from the small roles to the compute warps at the start (setmaxnreg)
+// warps 0-7 compute, 8 issues the contractions, 9 loads, 10-11 idle, 12-15 write the results
 constexpr int kBwdThreads = 512;
 constexpr int kWriterWarp0 = 12;
 constexpr int kWriterThreads = 128;
