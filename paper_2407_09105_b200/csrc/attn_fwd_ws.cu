@@ -183,7 +183,8 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
 
   float* s_invl = reinterpret_cast<float*>(smem + L::kInvL);
   // Register budget: 512 threads start with 128 each; every warpgroup changes its allowance at the
-  // top of its own branch.
+  // top of its own branch.  The two decreases free 128 * (88 + 32) = 15 360 registers without
+  // waiting for anything, the increases take 256 * 56 = 14 336: they cannot block for good.
   if ((warp >> 2) == (kFwsMmaWarp >> 2)) {
   setmaxnreg_dec<40>();
   if (warp == kFwsLoadWarp) {
