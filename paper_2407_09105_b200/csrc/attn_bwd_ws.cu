@@ -301,6 +301,10 @@ attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         tc_fence_after();
         issue_s(gs);
         issue_dp(gs);
+        // K and V are read for the last time by the unit's last S^T and dP^T, which are issued one
+        // step before its end: releasing them there lets the next unit's K and V arrive while this
+        // unit's last dV and dK still run
+        if (n_steps == 1 && leader) mma_commit(bar(kvKvEmpty));
         for (int s = 0; s < n_steps; ++s, ++gs) {
           const uint32_t tA = region_s(gs);
           const uint32_t doT_lo = desc_lo(sbase + L::kDo0 + (gs & 1) * L::kTileBytes, L::kBoxBytes);
@@ -339,11 +343,9 @@ attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           }
           __syncwarp();
           if (more) issue_dp(gs + 1);             // over P / dS(s), consumed just above
+          if (s + 2 == n_steps && leader) mma_commit(bar(kvKvEmpty));
         }
-        if (leader) {
-          mma_commit(bar(kvUnitDone));
-          mma_commit(bar(kvKvEmpty));
-        }
+        if (leader) mma_commit(bar(kvUnitDone));
         __syncwarp();
       }
     }

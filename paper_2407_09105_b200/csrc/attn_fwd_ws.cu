@@ -264,6 +264,9 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         tc_fence_after();
         issue_s(0, gk & 1);
         issue_s(1, gk & 1);
+        // the Q tiles are read for the last time by the unit's last S, issued one step before its
+        // end: releasing them there lets the next unit's Q arrive while the last P V still run
+        if (j0 + 1 == n_kv && leader) mma_commit(bar(fQEmpty));
         for (int j = j0; j < n_kv; ++j, ++gk) {
           const int st = gk & 1;
           const uint32_t v_lo =
@@ -289,10 +292,10 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                 tc_fence_after();
               }
               issue_s(t, (gk + 1) & 1);
+              if (t == 1 && j + 2 == n_kv && leader) mma_commit(bar(fQEmpty));
             }
           }
         }
-        if (leader) mma_commit(bar(fQEmpty));
         __syncwarp();
       }
     }
