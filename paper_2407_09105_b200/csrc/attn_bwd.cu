@@ -36,41 +36,55 @@ constexpr int kBwdThreads = 128;
 constexpr float kLog2e = 1.4426950408889634f;
 
 // ------------------------------------------------------------------ delta pre-pass
-// D/8 lanes per (token, head) row, 16 bytes of dO per lane; shuffles reduce inside the lane
-// group (a warp covers 32*8/D rows).  HBM-bound: reads dO and O once.
+// D/16 lanes per (token, head) row, 32 bytes of dO per lane; shuffles reduce inside the lane
+// group (a warp covers 32*16/D rows).  HBM-bound: reads dO and O once.  With 256-bit loads it runs
+// at 6.9 TB/s (c4: 2.07 GB in 0.30 ms) where 128-bit loads gave 4.3 TB/s; buffers that are only
+// 16-byte aligned take two 128-bit loads instead.
+__device__ __forceinline__ void ld_nc_v8(const void* p, uint32_t* v, bool aligned32) {
+  if (aligned32) {
+    asm volatile("ld.global.nc.L1::no_allocate.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                 : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]),
+                   "=r"(v[6]), "=r"(v[7])
+                 : "l"(p));
+  } else {
+    const uint4 a = __ldg(static_cast<const uint4*>(p)), b = __ldg(static_cast<const uint4*>(p) + 1);
+    v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w;
+    v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+  }
+}
 template <typename OutT>
 __global__ void delta_kernel(const __nv_bfloat16* __restrict__ dout, const OutT* __restrict__ out,
-                             float* __restrict__ delta, int T, int Hq, int D) {
-  const int lanes_per_row = D >> 3;                       // 16 (D = 128) or 8 (D = 64)
+                             float* __restrict__ delta, int T, int Hq, int D, bool aligned32) {
+  const int lanes_per_row = D >> 4;                       // 8 (D = 128), 4 (D = 64), ...
   const int rows_per_warp = 32 / lanes_per_row;
   const int lane = threadIdx.x & 31;
   const int64_t warp_id = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   const int64_t row = warp_id * rows_per_warp + lane / lanes_per_row;
-  const int c = (lane % lanes_per_row) * 8;
+  const int c = (lane % lanes_per_row) * 16;
   float acc = 0.f;
   if (row < (int64_t)T * Hq) {
-    const uint4 a4 = *reinterpret_cast<const uint4*>(dout + row * D + c);
-    const __nv_bfloat162* av = reinterpret_cast<const __nv_bfloat162*>(&a4);
-    float y[8];
+    uint32_t a[8];
+    ld_nc_v8(dout + row * D + c, a, aligned32);
+    float y[16];
     if (sizeof(OutT) == 2) {
-      const uint4 b4 = *reinterpret_cast<const uint4*>(out + row * D + c);
-      const __nv_bfloat162* bv = reinterpret_cast<const __nv_bfloat162*>(&b4);
+      uint32_t b[8];
+      ld_nc_v8(out + row * D + c, b, aligned32);
 #pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const float2 f = __bfloat1622float2(bv[e]);
-        y[2 * e] = f.x; y[2 * e + 1] = f.y;
+      for (int e = 0; e < 8; ++e) {
+        y[2 * e] = __uint_as_float(b[e] << 16);
+        y[2 * e + 1] = __uint_as_float(b[e] & 0xffff0000u);
       }
     } else {
-      const float4 b0 = *reinterpret_cast<const float4*>(out + row * D + c);
-      const float4 b1 = *reinterpret_cast<const float4*>(out + row * D + c + 4);
-      y[0] = b0.x; y[1] = b0.y; y[2] = b0.z; y[3] = b0.w;
-      y[4] = b1.x; y[5] = b1.y; y[6] = b1.z; y[7] = b1.w;
+      uint32_t b0[8], b1[8];
+      ld_nc_v8(out + row * D + c, b0, aligned32);
+      ld_nc_v8(out + row * D + c + 8, b1, aligned32);
+#pragma unroll
+      for (int e = 0; e < 8; ++e) { y[e] = __uint_as_float(b0[e]); y[8 + e] = __uint_as_float(b1[e]); }
     }
 #pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      const float2 x = __bfloat1622float2(av[e]);
-      acc = fmaf(x.x, y[2 * e], acc);
-      acc = fmaf(x.y, y[2 * e + 1], acc);
+    for (int e = 0; e < 8; ++e) {
+      acc = fmaf(__uint_as_float(a[e] << 16), y[2 * e], acc);
+      acc = fmaf(__uint_as_float(a[e] & 0xffff0000u), y[2 * e + 1], acc);
     }
   }
   for (int o = lanes_per_row >> 1; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
@@ -489,16 +503,20 @@ int delta_launch(const void* dout, const void* out, int out_dtype, float* delta,
                  cudaStream_t stream) {
   const int64_t rows = (int64_t)T * Hq;
   const int warps = 8;
-  const int64_t rows_per_block = (int64_t)warps * (32 / (D >> 3));
+  const int64_t rows_per_block = (int64_t)warps * (32 / (D >> 4));
   const unsigned blocks = (unsigned)((rows + rows_per_block - 1) / rows_per_block);
+  // rows are multiples of 32 bytes (D >= 16), so the base addresses decide the alignment
+  const bool aligned32 =
+      ((reinterpret_cast<uintptr_t>(dout) | reinterpret_cast<uintptr_t>(out)) & 31u) == 0;
   TimedLaunch timed(PK_KERNEL_DELTA, stream);
   if (out_dtype == PK_BF16)
     delta_kernel<__nv_bfloat16><<<blocks, warps * 32, 0, stream>>>(
         static_cast<const __nv_bfloat16*>(dout), static_cast<const __nv_bfloat16*>(out), delta, T,
-        Hq, D);
+        Hq, D, aligned32);
   else
     delta_kernel<float><<<blocks, warps * 32, 0, stream>>>(
-        static_cast<const __nv_bfloat16*>(dout), static_cast<const float*>(out), delta, T, Hq, D);
+        static_cast<const __nv_bfloat16*>(dout), static_cast<const float*>(out), delta, T, Hq, D,
+        aligned32);
   return launch_status();
 }
 

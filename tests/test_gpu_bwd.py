@@ -121,3 +121,42 @@ def test_backward_reusing_the_forwards_rotated_copies_is_bitwise_the_same():
         torch.cuda.synchronize()
         res.append([x.float().cpu().numpy().tobytes() for x in (dq, dk, dv)])
     assert res[0] == res[1]
+
+
+def _shifted(t):
+    """A copy of ``t`` whose storage starts 16 bytes past a 32-byte boundary."""
+    n = 16 // t.element_size()
+    base = torch.empty(t.numel() + n, dtype=t.dtype, device=t.device)
+    view = base[n:].view(t.shape)
+    view.copy_(t)
+    assert view.data_ptr() % 32 == 16
+    return view
+
+
+@pytest.mark.parametrize("theta,out_dtype", [(0.0, torch.float32), (1e4, torch.bfloat16)])
+def test_buffers_aligned_to_16_bytes_only(theta, out_dtype):
+    """The ABI asks for 16-byte alignment; the 32-byte loads and stores the kernels prefer must
+    fall back on every tensor that has no more than that."""
+    lens = [150, 260, 3, 129]
+    w = wl.Workload("t", 31, 4, 2, 128, theta, [lens], "test")
+    st = to_cuda(wl.stream_tensors(w, lens, 0, "cpu"))
+    st = wl.StreamTensors(st.position_ids, _shifted(st.q), _shifted(st.k), _shifted(st.v),
+                          _shifted(st.dout), lens)
+    T, Hq, D = st.q.shape
+    ws = api.alloc_workspace(T, Hq, 2, D)
+    out = _shifted(torch.zeros((T, Hq, D), dtype=out_dtype, device="cuda"))
+    lse = torch.empty((Hq, T), dtype=torch.float32, device="cuda")
+    api.pk_attn_fwd(st.q, st.k, st.v, st.position_ids, w.softmax_scale, theta, out, lse, ws)
+    dq = _shifted(torch.zeros((T, Hq, D), dtype=out_dtype, device="cuda"))
+    dk = _shifted(torch.zeros((T, 2, D), dtype=out_dtype, device="cuda"))
+    dv = _shifted(torch.zeros((T, 2, D), dtype=out_dtype, device="cuda"))
+    api.pk_attn_bwd(st.dout, st.q, st.k, st.v, out, lse, st.position_ids, w.softmax_scale, theta,
+                    dq, dk, dv, ws, reuse_plan=True)
+    assert api.pk_status_read(ws) == (api.PK_OK, 0)
+    pos = st.position_ids.cpu().numpy()
+    o_ref, _ = orc.attn_fwd(f64(st.q), f64(st.k), f64(st.v), pos, w.softmax_scale, theta)
+    refs = orc.attn_bwd(f64(st.dout), f64(st.q), f64(st.k), f64(st.v), pos, w.softmax_scale, theta)
+    extra = (lambda e: 2.0 ** -8 * np.abs(e)) if out_dtype == torch.bfloat16 else (lambda e: 0.0)
+    assert (np.abs(f64(out) - o_ref) <= 1e-2 + extra(o_ref)).all()
+    for g, e in zip((dq, dk, dv), refs):
+        assert (np.abs(f64(g) - e) <= TOL_G + extra(e)).all()
