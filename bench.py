@@ -500,8 +500,9 @@ def main():
     ms_step = replicas.max_over_ranks(e0.elapsed_time(e1), dist, "cuda") / args.steps
     fwd_ms = float(np.mean([a.elapsed_time(b) for a, b in kev[api.PK_KERNEL_FWD]]))
     bwd_ms = float(np.mean([a.elapsed_time(b) for a, b in kev[api.PK_KERNEL_BWD]]))
-    # two backward kernels unless the in-tile RoPE kernels run (RoPE with head_dim != 128)
-    split = theta <= 0 or D == 128
+    # two backward kernels (dK/dV, dQ): bench.py never selects the in-tile RoPE mode, whose single
+    # backward kernel would be timed as PK_KERNEL_BWD alone
+    split = True
     dq_ms = float(np.mean([a.elapsed_time(b) for a, b in kev[api.PK_KERNEL_BWD_DQ]])) if split else 0.0
 
     flops_step = w.useful_flops_fwd + w.useful_flops_bwd
